@@ -1,0 +1,340 @@
+// C ABI: argument validation, workspace carving and launch sequencing.  No compute here.
+#include <mutex>
+
+#include "common.cuh"
+
+namespace moe {
+
+int sm_count()
+{
+    static int cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
+        return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+static thread_local int g_last_launches = 0;
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static moe_status_t check_config(const moe_config_t *c)
+{
+    if (!c)
+        return MOE_ERR_INVALID_ARG;
+    if (c->hidden < 32 || c->hidden % 32 || c->inter < 32 || c->inter % 32)
+        return MOE_ERR_INVALID_ARG;
+    if (c->shared_inter < 0 || c->shared_inter % 32)
+        return MOE_ERR_INVALID_ARG;
+    if (c->n_experts < 1 || c->n_experts > MOE_MAX_EXPERTS)
+        return MOE_ERR_INVALID_ARG;
+    if (c->top_k < 1 || c->top_k > MOE_MAX_TOPK || c->top_k > c->n_experts)
+        return MOE_ERR_INVALID_ARG;
+    if (c->score_fn != MOE_SCORE_SOFTMAX && c->score_fn != MOE_SCORE_SIGMOID)
+        return MOE_ERR_INVALID_ARG;
+    return MOE_OK;
+}
+
+static moe_status_t check_tokens(const moe_config_t *c, int64_t T)
+{
+    if (T < 1 || T * c->top_k >= (1 << 24))
+        return MOE_ERR_INVALID_ARG;
+    return MOE_OK;
+}
+
+// The kernels are built for sm_100a only.
+static moe_status_t check_device()
+{
+    static int ok[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    if (dev < 0 || dev >= 64)
+        return MOE_ERR_UNSUPPORTED;
+    if (ok[dev] == 0) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+            return MOE_ERR_CUDA;
+        ok[dev] = major == 10 ? 1 : -1;
+    }
+    return ok[dev] == 1 ? MOE_OK : MOE_ERR_UNSUPPORTED;
+}
+
+static bool weights_ok(const moe_config_t *c, const moe_weights_t *w, bool need_router,
+                       bool need_experts)
+{
+    if (!w)
+        return false;
+    if (need_router) {
+        if (!w->w_router || !aligned16(w->w_router))
+            return false;
+        if (c->shared_inter > 0 && c->shared_gate && (!w->w_shared_gate || !aligned16(w->w_shared_gate)))
+            return false;
+    }
+    if (need_experts) {
+        if (!w->w_gate || !w->w_up || !w->w_down)
+            return false;
+        if (!aligned16(w->w_gate) || !aligned16(w->w_up) || !aligned16(w->w_down))
+            return false;
+        if (c->shared_inter > 0) {
+            if (!w->ws_gate || !w->ws_up || !w->ws_down)
+                return false;
+            if (!aligned16(w->ws_gate) || !aligned16(w->ws_up) || !aligned16(w->ws_down))
+                return false;
+        }
+    }
+    return true;
+}
+
+#define MOE_TRY_LAUNCH(expr)            \
+    do {                                \
+        if ((expr) != cudaSuccess)      \
+            return MOE_ERR_CUDA;        \
+        ++launches;                     \
+    } while (0)
+
+static moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x,
+                            int T, const int32_t *offsets, const int32_t *perm,
+                            __nv_bfloat16 *y, __nv_bfloat16 *shared_y, char *ws,
+                            const Workspace &L, cudaStream_t s, int &launches)
+{
+    const bool with_shared = shared_y != nullptr && c.shared_inter > 0;
+    PlanView plan{reinterpret_cast<int32_t *>(ws + L.plan_header),
+                  reinterpret_cast<Segment *>(ws + L.plan_routed),
+                  reinterpret_cast<Segment *>(ws + L.plan_shared)};
+    __nv_bfloat16 *h = reinterpret_cast<__nv_bfloat16 *>(ws + L.h);
+    __nv_bfloat16 *hs = reinterpret_cast<__nv_bfloat16 *>(ws + L.h_shared);
+    MOE_TRY_LAUNCH(launch_plan(c, T, offsets, with_shared,
+                               reinterpret_cast<int32_t *>(ws + L.status), plan, s));
+    MOE_TRY_LAUNCH(launch_ffn_stream_gateup(c, w, x, T, perm, plan, with_shared, h, hs, s));
+    MOE_TRY_LAUNCH(launch_ffn_stream_down(c, w, T, plan, with_shared, h, hs, y, shared_y, s));
+    return MOE_OK;
+}
+
+}  // namespace moe
+
+using namespace moe;
+
+extern "C" {
+
+size_t moe_workspace_bytes(const moe_config_t *cfg, int32_t max_tokens)
+{
+    if (check_config(cfg) != MOE_OK || check_tokens(cfg, max_tokens) != MOE_OK)
+        return 0;
+    return workspace_layout(*cfg, max_tokens).total;
+}
+
+moe_status_t moe_router_logits(const moe_config_t *cfg, const moe_weights_t *w, const void *x,
+                               int32_t T, float *logits, float *shared_scale, void *stream)
+{
+    moe_status_t st = check_config(cfg);
+    if (st != MOE_OK)
+        return st;
+    if ((st = check_tokens(cfg, T)) != MOE_OK)
+        return st;
+    if (!weights_ok(cfg, w, true, false) || !x || !logits || !aligned16(x) || !aligned16(logits))
+        return MOE_ERR_INVALID_ARG;
+    if ((st = check_device()) != MOE_OK)
+        return st;
+    int launches = 0;
+    MOE_TRY_LAUNCH(launch_router_logits(*cfg, *w, static_cast<const __nv_bfloat16 *>(x), T, logits,
+                                        shared_scale, static_cast<cudaStream_t>(stream)));
+    return MOE_OK;
+}
+
+moe_status_t moe_route_topk(const moe_config_t *cfg, const float *logits, int32_t T,
+                            int32_t *topk_idx, float *topk_w, void *stream)
+{
+    moe_status_t st = check_config(cfg);
+    if (st != MOE_OK)
+        return st;
+    if ((st = check_tokens(cfg, T)) != MOE_OK)
+        return st;
+    if (!logits || !topk_idx || !topk_w || !aligned16(logits) || !aligned16(topk_idx) ||
+        !aligned16(topk_w))
+        return MOE_ERR_INVALID_ARG;
+    if ((st = check_device()) != MOE_OK)
+        return st;
+    int launches = 0;
+    MOE_TRY_LAUNCH(launch_route_topk(*cfg, logits, T, topk_idx, topk_w,
+                                     static_cast<cudaStream_t>(stream)));
+    return MOE_OK;
+}
+
+moe_status_t moe_permute(const moe_config_t *cfg, const int32_t *topk_idx, int32_t T,
+                         int32_t *counts, int32_t *offsets, int32_t *perm, int32_t *inv_perm,
+                         int32_t *active, int32_t *n_active, void *stream)
+{
+    moe_status_t st = check_config(cfg);
+    if (st != MOE_OK)
+        return st;
+    if ((st = check_tokens(cfg, T)) != MOE_OK)
+        return st;
+    if (!topk_idx || !counts || !offsets || !perm || !inv_perm || !active || !n_active)
+        return MOE_ERR_INVALID_ARG;
+    if (!aligned16(topk_idx) || !aligned16(perm) || !aligned16(inv_perm))
+        return MOE_ERR_INVALID_ARG;
+    if ((st = check_device()) != MOE_OK)
+        return st;
+    int launches = 0;
+    MOE_TRY_LAUNCH(launch_permute(*cfg, topk_idx, T, counts, offsets, perm, inv_perm, active,
+                                  n_active, static_cast<cudaStream_t>(stream)));
+    return MOE_OK;
+}
+
+moe_status_t moe_grouped_swiglu(const moe_config_t *cfg, const moe_weights_t *w, const void *x,
+                                int32_t T, const int32_t *offsets, const int32_t *perm,
+                                const int32_t *active, const int32_t *n_active, void *y,
+                                void *shared_y, void *ws, size_t ws_bytes, void *stream)
+{
+    moe_status_t st = check_config(cfg);
+    if (st != MOE_OK)
+        return st;
+    if ((st = check_tokens(cfg, T)) != MOE_OK)
+        return st;
+    if (!weights_ok(cfg, w, false, true) || !x || !offsets || !perm || !active || !n_active || !y ||
+        !ws)
+        return MOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y) || !aligned16(ws) || (shared_y && !aligned16(shared_y)))
+        return MOE_ERR_INVALID_ARG;
+    const Workspace L = workspace_layout(*cfg, T);
+    if (ws_bytes < L.total)
+        return MOE_ERR_WORKSPACE;
+    if ((st = check_device()) != MOE_OK)
+        return st;
+    int launches = 0;
+    return run_ffn(*cfg, *w, static_cast<const __nv_bfloat16 *>(x), T, offsets, perm,
+                   static_cast<__nv_bfloat16 *>(y), static_cast<__nv_bfloat16 *>(shared_y),
+                   static_cast<char *>(ws), L, static_cast<cudaStream_t>(stream), launches);
+}
+
+moe_status_t moe_combine(const moe_config_t *cfg, const void *y, const int32_t *inv_perm,
+                         const float *topk_w, const void *shared_y, const float *shared_scale,
+                         int32_t T, void *out, void *stream)
+{
+    moe_status_t st = check_config(cfg);
+    if (st != MOE_OK)
+        return st;
+    if ((st = check_tokens(cfg, T)) != MOE_OK)
+        return st;
+    if (!y || !inv_perm || !topk_w || !out || !aligned16(y) || !aligned16(out) ||
+        (shared_y && !aligned16(shared_y)))
+        return MOE_ERR_INVALID_ARG;
+    if ((st = check_device()) != MOE_OK)
+        return st;
+    int launches = 0;
+    MOE_TRY_LAUNCH(launch_combine(*cfg, static_cast<const __nv_bfloat16 *>(y), inv_perm, topk_w,
+                                  static_cast<const __nv_bfloat16 *>(shared_y), shared_scale, T,
+                                  static_cast<__nv_bfloat16 *>(out),
+                                  static_cast<cudaStream_t>(stream)));
+    return MOE_OK;
+}
+
+moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, const void *x,
+                              int32_t B, int32_t gamma, void *out, const moe_debug_out_t *dbg,
+                              void *ws, size_t ws_bytes, void *stream)
+{
+    g_last_launches = 0;
+    moe_status_t st = check_config(cfg);
+    if (st != MOE_OK)
+        return st;
+    if (B < 1 || gamma < 0)
+        return MOE_ERR_INVALID_ARG;
+    const int64_t T64 = (int64_t)B * ((int64_t)gamma + 1);
+    if ((st = check_tokens(cfg, T64)) != MOE_OK)
+        return st;
+    const int T = (int)T64;
+    if (!weights_ok(cfg, w, true, true) || !x || !out || !ws || !aligned16(x) || !aligned16(out) ||
+        !aligned16(ws))
+        return MOE_ERR_INVALID_ARG;
+    const Workspace L = workspace_layout(*cfg, T);
+    if (ws_bytes < L.total)
+        return MOE_ERR_WORKSPACE;
+    if ((st = check_device()) != MOE_OK)
+        return st;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char *base = static_cast<char *>(ws);
+    const __nv_bfloat16 *xb = static_cast<const __nv_bfloat16 *>(x);
+    float *logits = reinterpret_cast<float *>(base + L.logits);
+    int32_t *topk_idx = reinterpret_cast<int32_t *>(base + L.topk_idx);
+    float *topk_w = reinterpret_cast<float *>(base + L.topk_w);
+    float *shared_scale = reinterpret_cast<float *>(base + L.shared_scale);
+    int32_t *counts = reinterpret_cast<int32_t *>(base + L.counts);
+    int32_t *offsets = reinterpret_cast<int32_t *>(base + L.offsets);
+    int32_t *active = reinterpret_cast<int32_t *>(base + L.active);
+    int32_t *n_active = reinterpret_cast<int32_t *>(base + L.n_active);
+    int32_t *perm = reinterpret_cast<int32_t *>(base + L.perm);
+    int32_t *inv_perm = reinterpret_cast<int32_t *>(base + L.inv_perm);
+    __nv_bfloat16 *y = reinterpret_cast<__nv_bfloat16 *>(base + L.y);
+    const bool has_shared = cfg->shared_inter > 0;
+    const bool gated = has_shared && cfg->shared_gate;
+    __nv_bfloat16 *ys = has_shared ? reinterpret_cast<__nv_bfloat16 *>(base + L.y_shared) : nullptr;
+
+    int launches = 0;
+    MOE_TRY_LAUNCH(launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s));
+    MOE_TRY_LAUNCH(launch_route_topk(*cfg, logits, T, topk_idx, topk_w, s));
+    MOE_TRY_LAUNCH(launch_permute(*cfg, topk_idx, T, counts, offsets, perm, inv_perm, active,
+                                  n_active, s));
+    st = run_ffn(*cfg, *w, xb, T, offsets, perm, y, ys, base, L, s, launches);
+    if (st != MOE_OK)
+        return st;
+    MOE_TRY_LAUNCH(launch_combine(*cfg, y, inv_perm, topk_w, ys, gated ? shared_scale : nullptr, T,
+                                  static_cast<__nv_bfloat16 *>(out), s));
+    g_last_launches = launches;
+
+    if (dbg) {
+        const size_t A = (size_t)T * cfg->top_k, E = cfg->n_experts;
+        struct Copy {
+            void *dst;
+            const void *src;
+            size_t bytes;
+        } copies[] = {
+            {dbg->logits, logits, (size_t)T * E * 4}, {dbg->topk_idx, topk_idx, A * 4},
+            {dbg->topk_w, topk_w, A * 4},             {dbg->counts, counts, E * 4},
+            {dbg->offsets, offsets, (E + 1) * 4},     {dbg->perm, perm, A * 4},
+            {dbg->inv_perm, inv_perm, A * 4},         {dbg->active, active, E * 4},
+            {dbg->n_active, n_active, 4},
+        };
+        for (const Copy &cp : copies)
+            if (cp.dst && cudaMemcpyAsync(cp.dst, cp.src, cp.bytes, cudaMemcpyDeviceToDevice, s) !=
+                              cudaSuccess)
+                return MOE_ERR_CUDA;
+    }
+    return MOE_OK;
+}
+
+moe_status_t moe_check(void *ws, void *stream)
+{
+    if (!ws)
+        return MOE_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    int32_t word = 0;
+    if (cudaMemcpy(&word, ws, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    return word == 0 ? MOE_OK : MOE_ERR_TIMEOUT;
+}
+
+int32_t moe_last_launch_count(void) { return g_last_launches; }
+
+const char *moe_status_string(moe_status_t s)
+{
+    switch (s) {
+    case MOE_OK: return "ok";
+    case MOE_ERR_INVALID_ARG: return "invalid argument";
+    case MOE_ERR_UNSUPPORTED: return "unsupported (needs an sm_100a GPU)";
+    case MOE_ERR_WORKSPACE: return "workspace too small";
+    case MOE_ERR_CUDA: return "CUDA runtime error";
+    case MOE_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

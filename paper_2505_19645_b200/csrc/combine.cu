@@ -1,0 +1,79 @@
+// Gate-weighted combine: out[t] = sum_j w[t,j] * y[inv_perm[t*K+j]] + s[t] * shared_y[t].
+// Gather form (each output row is summed in slot order by one owner), so the result does
+// not depend on scheduling; 128-bit loads and stores.
+#include "common.cuh"
+
+namespace moe {
+
+constexpr int CB_THREADS = 256;
+
+__global__ void __launch_bounds__(CB_THREADS)
+combine_kernel(const __nv_bfloat16 *__restrict__ y, const int32_t *__restrict__ inv_perm,
+               const float *__restrict__ topk_w, const __nv_bfloat16 *__restrict__ shared_y,
+               const float *__restrict__ shared_scale, int T, int H, int k,
+               __nv_bfloat16 *__restrict__ out)
+{
+    const int vec_per_row = H >> 3;
+    const size_t total = (size_t)T * vec_per_row;
+    for (size_t i = blockIdx.x * (size_t)CB_THREADS + threadIdx.x; i < total;
+         i += (size_t)gridDim.x * CB_THREADS) {
+        const int t = (int)(i / vec_per_row);
+        const int h = (int)(i - (size_t)t * vec_per_row) << 3;
+        float acc[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            acc[q] = 0.f;
+        for (int j = 0; j < k; ++j) {
+            const int row = inv_perm[(size_t)t * k + j];
+            const float w = topk_w[(size_t)t * k + j];
+            const uint4 v = *reinterpret_cast<const uint4 *>(y + (size_t)row * H + h);
+            acc[0] = fmaf(w, bf16_lo(v.x), acc[0]);
+            acc[1] = fmaf(w, bf16_hi(v.x), acc[1]);
+            acc[2] = fmaf(w, bf16_lo(v.y), acc[2]);
+            acc[3] = fmaf(w, bf16_hi(v.y), acc[3]);
+            acc[4] = fmaf(w, bf16_lo(v.z), acc[4]);
+            acc[5] = fmaf(w, bf16_hi(v.z), acc[5]);
+            acc[6] = fmaf(w, bf16_lo(v.w), acc[6]);
+            acc[7] = fmaf(w, bf16_hi(v.w), acc[7]);
+        }
+        if (shared_y) {
+            const float s = shared_scale ? shared_scale[t] : 1.0f;
+            const uint4 v = *reinterpret_cast<const uint4 *>(shared_y + (size_t)t * H + h);
+            acc[0] = fmaf(s, bf16_lo(v.x), acc[0]);
+            acc[1] = fmaf(s, bf16_hi(v.x), acc[1]);
+            acc[2] = fmaf(s, bf16_lo(v.y), acc[2]);
+            acc[3] = fmaf(s, bf16_hi(v.y), acc[3]);
+            acc[4] = fmaf(s, bf16_lo(v.z), acc[4]);
+            acc[5] = fmaf(s, bf16_hi(v.z), acc[5]);
+            acc[6] = fmaf(s, bf16_lo(v.w), acc[6]);
+            acc[7] = fmaf(s, bf16_hi(v.w), acc[7]);
+        }
+        uint4 o;
+        __nv_bfloat162 p;
+        p = __floats2bfloat162_rn(acc[0], acc[1]);
+        o.x = *reinterpret_cast<uint32_t *>(&p);
+        p = __floats2bfloat162_rn(acc[2], acc[3]);
+        o.y = *reinterpret_cast<uint32_t *>(&p);
+        p = __floats2bfloat162_rn(acc[4], acc[5]);
+        o.z = *reinterpret_cast<uint32_t *>(&p);
+        p = __floats2bfloat162_rn(acc[6], acc[7]);
+        o.w = *reinterpret_cast<uint32_t *>(&p);
+        *reinterpret_cast<uint4 *>(out + (size_t)t * H + h) = o;
+    }
+}
+
+cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, const int32_t *inv_perm,
+                           const float *topk_w, const __nv_bfloat16 *shared_y,
+                           const float *shared_scale, int T, __nv_bfloat16 *out, cudaStream_t s)
+{
+    const size_t total = (size_t)T * (c.hidden >> 3);
+    size_t blocks = (total + CB_THREADS - 1) / CB_THREADS;
+    const size_t cap = (size_t)sm_count() * 8;
+    if (blocks > cap)
+        blocks = cap;
+    combine_kernel<<<(unsigned)blocks, CB_THREADS, 0, s>>>(y, inv_perm, topk_w, shared_y,
+                                                          shared_scale, T, c.hidden, c.top_k, out);
+    return cudaGetLastError();
+}
+
+}  // namespace moe

@@ -1,0 +1,75 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every declared symbol, and
+rejects bad arguments on the host before anything could be launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2505_19645_b200 import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in os.listdir(inc):
+        if not f.endswith(".h"):
+            continue
+        text = open(os.path.join(inc, f)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        for m in re.finditer(r"\b(moe_[a-z_0-9]+)\s*\(", text):
+            names.add(m.group(1))
+    return sorted(names)
+
+
+def test_library_loads_and_exports_every_declared_symbol():
+    from paper_2505_19645_b200 import api
+
+    lib = api.load_library()
+    declared = _declared_functions()
+    assert len(declared) >= 9
+    for name in declared:
+        assert hasattr(lib, name), "missing export " + name
+    assert sorted(set(api.EXPORTS) - set(declared)) == []
+
+
+def test_status_strings():
+    from paper_2505_19645_b200 import api
+
+    assert api.status_string(0) == "ok"
+    assert "workspace" in api.status_string(3)
+
+
+def test_workspace_bytes_and_host_side_validation():
+    from paper_2505_19645_b200 import api
+
+    lib = api.load_library()
+    shape = wl.CONFIGS["qwen1.5-moe-a2.7b"]
+    cfg = api.make_config(shape)
+    n1, n2 = api.moe_workspace_bytes(cfg, 1), api.moe_workspace_bytes(cfg, 640)
+    # at least h [A,I], y [A,H], shared h and y
+    assert n2 > 640 * (4 * (1408 + 2048) + 5632 + 2048) * 2 and n1 < n2
+    assert api.moe_workspace_bytes(cfg, 0) == 0
+    bad = api.make_config(wl.small_shape("b", 64, 4, 5, 64))
+    assert api.moe_workspace_bytes(bad, 8) == 0
+    bad = api.make_config(wl.small_shape("b", 64, 600, 2, 64))
+    assert api.moe_workspace_bytes(bad, 8) == 0
+    # null pointers are refused with MOE_ERR_INVALID_ARG without touching a device
+    w = api.CWeights()
+    st = lib.moe_verify_layer(ctypes.byref(cfg), ctypes.byref(w), None, 1, 0, None, None, None, 0, None)
+    assert st == 1
+    st = lib.moe_route_topk(ctypes.byref(cfg), None, 4, None, None, None)
+    assert st == 1
+    st = lib.moe_permute(ctypes.byref(cfg), None, 4, None, None, None, None, None, None, None)
+    assert st == 1
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    from paper_2505_19645_b200 import api
+
+    monkeypatch.setattr(api, "_lib", None)
+    monkeypatch.setattr(api, "LIB_PATH", os.path.join(ROOT, "no_such_dir", "libmoe_verify.so"))
+    with pytest.raises(ImportError):
+        api.load_library()
