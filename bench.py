@@ -1,0 +1,426 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE verify layer (one pass of the whole hot path per step).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--config NAME] [--B B] [--gamma G] [--no-sweep]
+
+Prints ONE JSON line.  Default workload: the Qwen1.5-MoE-A2.7B-shaped layer at B=32
+sequences x (gamma=3)+1 tokens; the (B, gamma) grid of that shape is swept as well and
+reported under "sweep" (layer time, tokens/s, roofline fraction, T(B,gamma)/T(B,0)).
+Inputs are seeded and synthetic.  N > 1 runs N independent replicas (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2505_19645_b200 import replicas, workloads as wl  # noqa: E402
+
+L2_FLUSH_BYTES = 512 << 20
+DEFAULT_CONFIG = "qwen1.5-moe-a2.7b"
+DEFAULT_B, DEFAULT_GAMMA = 32, 3
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+# ---- algorithmic bytes / flops (activated experts only) ---------------------------------
+
+def layer_bytes(shape, T, n_active):
+    H, E, I, Is = shape.hidden, shape.n_experts, shape.inter, shape.shared_inter
+    return n_active * 6 * H * I + 6 * H * Is + E * H * 4 + 2 * T * H * 2
+
+
+def layer_flops(shape, T):
+    H, E, k, I, Is = shape.hidden, shape.n_experts, shape.top_k, shape.inter, shape.shared_inter
+    return T * k * 6 * H * I + T * 6 * H * Is + 2 * T * H * E
+
+
+def gate_up_bytes(shape, T, n_active):
+    """Gate/up kernel: both projections of every activated expert, once, plus the tokens."""
+    H, I, Is = shape.hidden, shape.inter, shape.shared_inter
+    return n_active * 4 * H * I + 4 * H * Is + T * H * 2
+
+
+def gate_up_flops(shape, T):
+    return T * shape.top_k * 4 * shape.hidden * shape.inter + T * 4 * shape.hidden * shape.shared_inter
+
+
+def expected_active(E, k, T):
+    return E * (1.0 - ((E - k) / E) ** T)
+
+
+# ---- clocks -----------------------------------------------------------------------------
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+        self.skip = 0
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines[self.skip:]:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---- GPU arm ----------------------------------------------------------------------------
+
+class LayerRunner:
+    def __init__(self, shape, weights_dev, device):
+        from paper_2505_19645_b200 import api
+        self.api = api
+        self.shape = shape
+        self.cfg = api.make_config(shape)
+        self.cw = api.make_weights(weights_dev)
+        self.keep = weights_dev
+        self.device = device
+        self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+
+    def prepare(self, T):
+        self.ws = self.api.alloc_workspace(self.cfg, T, self.device)
+        self.out = torch.empty((T, self.shape.hidden), dtype=torch.bfloat16, device=self.device)
+
+    def step(self, x, B, gamma):
+        T = B * (gamma + 1)
+        self.api.moe_verify_layer(self.cfg, self.cw, x, B, gamma, self.out[:T], self.ws)
+
+    def flush_l2(self):
+        self.flush.zero_()
+
+    def time_steps(self, x, B, gamma, steps, warmup, stage=None):
+        """Cold-L2 timing of `steps` layer passes; returns per-step ms (whole layer) and, if
+        `stage` is given, per-step ms of that kernel."""
+        api = self.api
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(steps)]
+        kev = None
+        if stage is not None:
+            kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(steps)]
+            for a, b in kev:   # torch creates the CUDA event lazily on first record
+                a.record()
+                b.record()
+        for _ in range(warmup):
+            self.flush_l2()
+            self.step(x, B, gamma)
+        torch.cuda.synchronize()
+        for i in range(steps):
+            self.flush_l2()
+            if kev is not None:
+                api.moe_profile_stage(stage, kev[i][0], kev[i][1])
+            ev[i][0].record()
+            self.step(x, B, gamma)
+            ev[i][1].record()
+        if kev is not None:
+            api.moe_profile_stage(None)
+        torch.cuda.synchronize()
+        api.moe_check(self.ws)
+        layer_ms = [a.elapsed_time(b) for a, b in ev]
+        kern_ms = [a.elapsed_time(b) for a, b in kev] if kev is not None else None
+        return layer_ms, kern_ms
+
+    def n_active(self, x, B, gamma):
+        dbg = {"n_active": torch.zeros(1, dtype=torch.int32, device=self.device)}
+        self.api.moe_verify_layer(self.cfg, self.cw, x, B, gamma, self.out[:B * (gamma + 1)],
+                                  self.ws, dbg)
+        torch.cuda.synchronize()
+        return int(dbg["n_active"].item())
+
+    def time_e2e(self, x_host_pinned, B, gamma, steps, warmup):
+        """Host buffers: H2D of the tokens, the layer, D2H of the result inside the timed region."""
+        T = x_host_pinned.shape[0]
+        x_dev = torch.empty((T, self.shape.hidden), dtype=torch.bfloat16, device=self.device)
+        out_host = torch.empty((T, self.shape.hidden), dtype=torch.bfloat16).pin_memory()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(steps)]
+        for i in range(warmup + steps):
+            self.flush_l2()
+            j = i - warmup
+            if j >= 0:
+                ev[j][0].record()
+            x_dev.copy_(x_host_pinned, non_blocking=True)
+            self.step(x_dev, B, gamma)
+            out_host.copy_(self.out[:T], non_blocking=True)
+            if j >= 0:
+                ev[j][1].record()
+        torch.cuda.synchronize()
+        ms = [a.elapsed_time(b) for a, b in ev]
+        nbytes = T * self.shape.hidden * 2
+        return ms, nbytes, nbytes
+
+
+def cpu_oracle_rate(shape, w_host, x_host, n_rows, repeats=1):
+    """Times the CPU oracle (as it stands) on a seeded sample of token rows; tokens/s."""
+    import numpy as np
+    import oracle
+    T = x_host.shape[0]
+    rng = np.random.default_rng(0)
+    rows = sorted(rng.choice(T, size=min(n_rows, T), replace=False).tolist())
+    cfg = dict(top_k=shape.top_k, score_fn=shape.score_fn, renormalize=shape.renormalize,
+               routed_scale=shape.routed_scale, shared_gate=shape.shared_gate)
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        oracle.verify_layer(x_host, w_host, cfg, rows=rows)
+        times.append(time.perf_counter() - t0)
+    # the router runs on all T rows (cheap); the FFNs on the sample
+    return len(rows) / min(times), len(rows), oracle.num_threads(), times
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores, same workload/metric/unit."""
+    rank, _, world = replicas.env_world()
+    if rank != 0:
+        return 0
+    shape = wl.CONFIGS[args.config]
+    T = args.B * (args.gamma + 1)
+    w = wl.make_weights(shape, wl.config_seed(args.config), "cpu")
+    x = wl.make_tokens(shape, T, wl.point_seed(args.config, args.B, args.gamma), "cpu")
+    import oracle
+    n_rows = min(T, max(1, oracle.num_threads()))
+    for _ in range(args.warmup):
+        cpu_oracle_rate(shape, w, x, n_rows)
+    rates = []
+    t_total = 0.0
+    for _ in range(args.steps):
+        r, n, cores, times = cpu_oracle_rate(shape, w, x, n_rows)
+        rates.append(r)
+        t_total += times[0]
+    value = n_rows * args.steps / t_total
+    sample = "%d seeded token rows of the T=%d batch per step" % (n_rows, T)
+    line = {
+        "impl": "reference", "metric": "moe_verify_layer_tokens_per_s", "value": value,
+        "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * t_total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded)",
+        "config": {"workload": workload_name(args), "config": args.config, "B": args.B,
+                   "gamma": args.gamma, "tokens": T},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def workload_name(args):
+    return "%s-shaped MoE FFN layer, B=%d, gamma=%d (T=%d tokens)" % (
+        args.config, args.B, args.gamma, args.B * (args.gamma + 1))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=wl.CONFIG_ORDER)
+    ap.add_argument("--B", type=int, default=DEFAULT_B)
+    ap.add_argument("--gamma", type=int, default=DEFAULT_GAMMA)
+    ap.add_argument("--zipf", type=float, default=None)
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep-steps", type=int, default=10)
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    if args.impl == "reference":
+        return run_reference(args)
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU fallback")
+    rank, world = replicas.init("nccl")
+    _, local_rank, _ = replicas.env_world()
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    peaks = load_peaks()
+
+    shape = wl.CONFIGS[args.config]
+    B, gamma = args.B, args.gamma
+    T = B * (gamma + 1)
+    w_dev = wl.make_weights(shape, wl.config_seed(args.config), device, zipf_s=args.zipf)
+    runner = LayerRunner(shape, w_dev, device)
+    max_T = T
+    if not args.no_sweep:
+        Bs, gs = wl.GRIDS[args.config]
+        max_T = max(max_T, max(Bs) * (max(gs) + 1))
+    runner.prepare(max_T)
+    seed = replicas.replica_seed(wl.point_seed(args.config, B, gamma), rank)
+    x = wl.make_tokens(shape, T, seed, device)
+    n_act = runner.n_active(x, B, gamma)
+    launches_per_step = runner.api.moe_last_launch_count()
+
+    # ---- headline: whole layer, inputs resident in HBM --------------------------------
+    # the sampler keeps running through the three measured loops (layer, kernel, end to end)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    runner.time_steps(x, B, gamma, 3, args.warmup)
+    replicas.barrier()
+    torch.cuda.synchronize()
+    sampler.skip = len(sampler.lines)
+    layer_ms, _ = runner.time_steps(x, B, gamma, args.steps, args.warmup)
+    torch.cuda.synchronize()
+    replicas.barrier()
+    ms_step_local = sum(layer_ms) / len(layer_ms)
+    value, ms_step = replicas.job_throughput(T, ms_step_local, device)
+
+    # ---- dominant kernel (gate/up) with its own event pair ----------------------------
+    _, kern_ms = runner.time_steps(x, B, gamma, args.steps, 3, stage="gate_up")
+    k_ms = sum(kern_ms) / len(kern_ms)
+    gu_bytes = gate_up_bytes(shape, T, n_act)
+    gu_flops = gate_up_flops(shape, T)
+    t_mem = gu_bytes / (peaks["hbm_gbs"] * 1e9)
+    t_flop = gu_flops / (peaks["bf16_tflops"] * 1e12)
+    if t_mem >= t_flop:
+        achieved = gu_bytes / (k_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"]}
+    else:
+        achieved = gu_flops / (k_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],
+                    "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"]}
+    roofline.update({"traffic": None, "kernel": "gate/up + SwiGLU", "kernel_ms": k_ms,
+                     "algorithmic_bytes": gu_bytes, "peak_source": peaks["source"]})
+
+    # whole-layer roofline: slower of activated-expert bytes over HBM and flops at tensor peak
+    def layer_roof_ms(Tn, nact):
+        return 1e3 * max(layer_bytes(shape, Tn, nact) / (peaks["hbm_gbs"] * 1e9),
+                         layer_flops(shape, Tn) / (peaks["bf16_tflops"] * 1e12))
+    layer_roof = {"roof_ms": layer_roof_ms(T, n_act), "frac": layer_roof_ms(T, n_act) / ms_step_local,
+                  "n_active": n_act, "bytes": layer_bytes(shape, T, n_act),
+                  "flops": layer_flops(shape, T), "median_ms": statistics.median(layer_ms),
+                  "min_ms": min(layer_ms)}
+
+    # ---- end to end with host buffers -------------------------------------------------
+    x_host = x.cpu().pin_memory()
+    e2e_ms, h2d, d2h = runner.time_e2e(x_host, B, gamma, args.steps, 3)
+    e2e_value, _ = replicas.job_throughput(T, sum(e2e_ms) / len(e2e_ms), device)
+    clocks = sampler.stop()
+
+    # ---- sweep of the config's (B, gamma) grid ----------------------------------------
+    sweep = []
+    if not args.no_sweep and rank == 0:
+        Bs, gs = wl.GRIDS[args.config]
+        for Bi in Bs:
+            base_ms = None
+            for gi in gs:
+                Ti = Bi * (gi + 1)
+                xi = wl.make_tokens(shape, Ti, wl.point_seed(args.config, Bi, gi), device)
+                na = runner.n_active(xi, Bi, gi)
+                ms, _ = runner.time_steps(xi, Bi, gi, args.sweep_steps, 3)
+                med = statistics.median(ms)
+                if gi == gs[0]:
+                    base_ms = med
+                roof = layer_roof_ms(Ti, na)
+                sweep.append({"B": Bi, "gamma": gi, "T": Ti, "us": round(med * 1e3, 2),
+                              "tokens_per_s": round(Ti / (med * 1e-3), 1), "n_active": na,
+                              "n_active_expected": round(expected_active(shape.n_experts, shape.top_k, Ti), 2),
+                              "roof_us": round(roof * 1e3, 2), "roof_frac": round(roof / med, 4),
+                              "ratio_vs_gamma0": round(med / base_ms, 4) if gs[0] == 0 else None})
+
+    # ---- CPU oracle beside it (rank 0, N = 1) -----------------------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        w_host = {k: (None if v is None else v.cpu()) for k, v in w_dev.items()}
+        import oracle
+        n_rows = min(T, 4 * oracle.num_threads())
+        x_cpu = x.cpu()
+        rate, n, cores, times = cpu_oracle_rate(shape, w_host, x_cpu, n_rows)
+        # repeat the sample until about 10 s of CPU work have been timed
+        reps = max(1, min(200, int(10.0 / max(times[0], 1e-3))))
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            cpu_oracle_rate(shape, w_host, x_cpu, n_rows)
+        dt = time.perf_counter() - t0
+        cpu = {"value": n * reps / dt, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+               "sample": "%d seeded token rows of the T=%d batch, %d passes, %.1f s"
+                         % (n, T, reps, dt)}
+
+    if rank == 0:
+        line = {
+            "metric": "moe_verify_layer_tokens_per_s", "value": value, "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic (seeded)",
+            "config": {"workload": workload_name(args), "config": args.config, "B": B,
+                       "gamma": gamma, "tokens": T, "zipf": args.zipf,
+                       "l2": "512 MiB buffer written between timed iterations",
+                       "parallelism": "replicas only"},
+            "roofline": roofline, "layer_roofline": layer_roof, "cpu_baseline": cpu,
+            "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+            "layer_us": ms_step * 1e3, "sweep": sweep,
+        }
+        print(json.dumps(line))
+    replicas.shutdown()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

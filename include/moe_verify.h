@@ -158,6 +158,22 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
  * invalid but the context stays usable), or MOE_ERR_CUDA. */
 moe_status_t moe_check(void *ws, void *stream);
 
+/* Measurement aid (no counterpart in the paper; its Sec. 3.3 model attributes the layer's
+ * time to weight loading, which the benchmark verifies per kernel).  Every following
+ * moe_verify_layer call of this thread records start_event before and stop_event after the
+ * kernel of the given stage on the call's stream.  Events are cudaEvent_t passed as void*,
+ * created and owned by the caller; stage < 0 switches the recording off. */
+typedef enum {
+    MOE_STAGE_ROUTER_LOGITS = 0,
+    MOE_STAGE_ROUTE_TOPK = 1,
+    MOE_STAGE_PERMUTE = 2,
+    MOE_STAGE_PLAN = 3,
+    MOE_STAGE_GATE_UP = 4,
+    MOE_STAGE_DOWN = 5,
+    MOE_STAGE_COMBINE = 6
+} moe_stage_t;
+moe_status_t moe_profile_stage(int32_t stage, void *start_event, void *stop_event);
+
 /* Number of kernels the last moe_verify_layer call on this thread enqueued. */
 int32_t moe_last_launch_count(void);
 

@@ -21,7 +21,10 @@ STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_UNSUPPORTED",
 
 EXPORTS = ["moe_workspace_bytes", "moe_router_logits", "moe_route_topk", "moe_permute",
            "moe_grouped_swiglu", "moe_combine", "moe_verify_layer", "moe_check",
-           "moe_last_launch_count", "moe_status_string"]
+           "moe_last_launch_count", "moe_status_string", "moe_profile_stage"]
+
+STAGES = {"router_logits": 0, "route_topk": 1, "permute": 2, "plan": 3, "gate_up": 4, "down": 5,
+          "combine": 6}
 
 
 class MoeError(RuntimeError):
@@ -83,6 +86,8 @@ def load_library():
                                      sz, vp]
     lib.moe_check.restype = i32
     lib.moe_check.argtypes = [vp, vp]
+    lib.moe_profile_stage.restype = i32
+    lib.moe_profile_stage.argtypes = [i32, vp, vp]
     lib.moe_last_launch_count.restype = i32
     lib.moe_last_launch_count.argtypes = []
     lib.moe_status_string.restype = ctypes.c_char_p
@@ -228,6 +233,18 @@ def moe_verify_layer(cfg, weights, x, B: int, gamma: int, out, ws, dbg: dict | N
 
 def moe_check(ws, stream=None):
     _check(load_library().moe_check(_ptr(ws), _stream_ptr(stream)), "moe_check")
+
+
+def moe_profile_stage(stage, start_event=None, stop_event=None):
+    """Record the two (already created) torch.cuda.Event objects around one kernel of every
+    following moe_verify_layer call of this thread; stage None / -1 switches it off."""
+    if stage is None or (isinstance(stage, int) and stage < 0):
+        _check(load_library().moe_profile_stage(-1, None, None), "moe_profile_stage")
+        return
+    sid = STAGES[stage] if isinstance(stage, str) else int(stage)
+    _check(load_library().moe_profile_stage(sid, ctypes.c_void_p(start_event.cuda_event),
+                                            ctypes.c_void_p(stop_event.cuda_event)),
+           "moe_profile_stage")
 
 
 def moe_last_launch_count() -> int:

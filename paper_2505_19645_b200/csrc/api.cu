@@ -99,6 +99,24 @@ static bool weights_ok(const moe_config_t *c, const moe_weights_t *w, bool need_
         ++launches;                     \
     } while (0)
 
+// Optional event pair around one stage of moe_verify_layer (see moe_profile_stage).
+struct StageProbe {
+    int stage = -1;
+    cudaEvent_t start = nullptr, stop = nullptr;
+};
+static thread_local StageProbe g_probe;
+static thread_local bool g_probe_armed = false;  // only moe_verify_layer arms it
+
+#define MOE_STAGE(stage_id, expr)                                             \
+    do {                                                                      \
+        const bool probe_ = g_probe_armed && g_probe.stage == (stage_id);     \
+        if (probe_ && cudaEventRecord(g_probe.start, s) != cudaSuccess)       \
+            return MOE_ERR_CUDA;                                              \
+        MOE_TRY_LAUNCH(expr);                                                 \
+        if (probe_ && cudaEventRecord(g_probe.stop, s) != cudaSuccess)        \
+            return MOE_ERR_CUDA;                                              \
+    } while (0)
+
 static moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x,
                             int T, const int32_t *offsets, const int32_t *perm,
                             __nv_bfloat16 *y, __nv_bfloat16 *shared_y, char *ws,
@@ -110,10 +128,12 @@ static moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const
                   reinterpret_cast<Segment *>(ws + L.plan_shared)};
     __nv_bfloat16 *h = reinterpret_cast<__nv_bfloat16 *>(ws + L.h);
     __nv_bfloat16 *hs = reinterpret_cast<__nv_bfloat16 *>(ws + L.h_shared);
-    MOE_TRY_LAUNCH(launch_plan(c, T, offsets, with_shared,
-                               reinterpret_cast<int32_t *>(ws + L.status), plan, s));
-    MOE_TRY_LAUNCH(launch_ffn_stream_gateup(c, w, x, T, perm, plan, with_shared, h, hs, s));
-    MOE_TRY_LAUNCH(launch_ffn_stream_down(c, w, T, plan, with_shared, h, hs, y, shared_y, s));
+    MOE_STAGE(MOE_STAGE_PLAN, launch_plan(c, T, offsets, with_shared,
+                                          reinterpret_cast<int32_t *>(ws + L.status), plan, s));
+    MOE_STAGE(MOE_STAGE_GATE_UP,
+              launch_ffn_stream_gateup(c, w, x, T, perm, plan, with_shared, h, hs, s));
+    MOE_STAGE(MOE_STAGE_DOWN,
+              launch_ffn_stream_down(c, w, T, plan, with_shared, h, hs, y, shared_y, s));
     return MOE_OK;
 }
 
@@ -278,15 +298,21 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
     __nv_bfloat16 *ys = has_shared ? reinterpret_cast<__nv_bfloat16 *>(base + L.y_shared) : nullptr;
 
     int launches = 0;
-    MOE_TRY_LAUNCH(launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s));
-    MOE_TRY_LAUNCH(launch_route_topk(*cfg, logits, T, topk_idx, topk_w, s));
-    MOE_TRY_LAUNCH(launch_permute(*cfg, topk_idx, T, counts, offsets, perm, inv_perm, active,
-                                  n_active, s));
+    struct Arm {
+        Arm() { g_probe_armed = true; }
+        ~Arm() { g_probe_armed = false; }
+    } arm;
+    MOE_STAGE(MOE_STAGE_ROUTER_LOGITS,
+              launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s));
+    MOE_STAGE(MOE_STAGE_ROUTE_TOPK, launch_route_topk(*cfg, logits, T, topk_idx, topk_w, s));
+    MOE_STAGE(MOE_STAGE_PERMUTE, launch_permute(*cfg, topk_idx, T, counts, offsets, perm, inv_perm,
+                                                active, n_active, s));
     st = run_ffn(*cfg, *w, xb, T, offsets, perm, y, ys, base, L, s, launches);
     if (st != MOE_OK)
         return st;
-    MOE_TRY_LAUNCH(launch_combine(*cfg, y, inv_perm, topk_w, ys, gated ? shared_scale : nullptr, T,
-                                  static_cast<__nv_bfloat16 *>(out), s));
+    MOE_STAGE(MOE_STAGE_COMBINE,
+              launch_combine(*cfg, y, inv_perm, topk_w, ys, gated ? shared_scale : nullptr, T,
+                             static_cast<__nv_bfloat16 *>(out), s));
     g_last_launches = launches;
 
     if (dbg) {
@@ -320,6 +346,16 @@ moe_status_t moe_check(void *ws, void *stream)
     if (cudaMemcpy(&word, ws, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess)
         return MOE_ERR_CUDA;
     return word == 0 ? MOE_OK : MOE_ERR_TIMEOUT;
+}
+
+moe_status_t moe_profile_stage(int32_t stage, void *start_event, void *stop_event)
+{
+    if (stage > MOE_STAGE_COMBINE || (stage >= 0 && (!start_event || !stop_event)))
+        return MOE_ERR_INVALID_ARG;
+    g_probe.stage = stage < 0 ? -1 : stage;
+    g_probe.start = static_cast<cudaEvent_t>(start_event);
+    g_probe.stop = static_cast<cudaEvent_t>(stop_event);
+    return MOE_OK;
 }
 
 int32_t moe_last_launch_count(void) { return g_last_launches; }
