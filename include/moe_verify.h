@@ -134,6 +134,35 @@ moe_status_t moe_grouped_swiglu(const moe_config_t *cfg, const moe_weights_t *w,
                                 const int32_t *active, const int32_t *n_active, void *y,
                                 void *shared_y, void *ws, size_t ws_bytes, void *stream);
 
+/* moe_grouped_swiglu without a caller-provided workspace (the paper has no counterpart; this
+ * is a packaging variant of the step above, same kernels, same results).
+ *
+ * Who needs it: callers that may not allocate device memory at the point where they run the
+ * layer -- an inference server that froze its memory plan at start-up, a plugin living inside
+ * another framework's allocator, a latency-critical loop that cannot risk the implicit
+ * device synchronisation of cudaMalloc/cudaFree -- and therefore cannot size and pass `ws`.
+ * The scratch (segment plan and the bf16 SwiGLU intermediates) lives in a fixed array of
+ * MOE_STATIC_SCRATCH_BYTES inside the library image; each GPU that loads the library holds it
+ * until the process exits.  The call itself allocates nothing, on host or device.
+ *
+ * Limit: the request must satisfy, with A = T*top_k and every term rounded up to 256 bytes,
+ *   256 + 64 + 16*(n_experts + A/32 + 1) + 16*ceil(T/32) + 2*A*inter + 2*T*shared_inter
+ *     <= MOE_STATIC_SCRATCH_BYTES,
+ * otherwise MOE_ERR_WORKSPACE is returned and nothing is launched (use moe_grouped_swiglu).
+ *
+ * Set-up: the first call on a device looks up the array's device address (once per device,
+ * with that device current).  Make that first call outside any stream capture.
+ * Sharing: every call on a device uses the same array and leaves its contents behind; the
+ * call clears what it needs cleared.  Two calls whose work overlaps on the GPU (different
+ * streams, or threads) race on it -- order them on one stream or with events.
+ * Arguments, results and error codes otherwise as for moe_grouped_swiglu. */
+#define MOE_STATIC_SCRATCH_BYTES (8u << 20)
+moe_status_t moe_grouped_swiglu_static(const moe_config_t *cfg, const moe_weights_t *w,
+                                       const void *x, int32_t T, const int32_t *offsets,
+                                       const int32_t *perm, const int32_t *active,
+                                       const int32_t *n_active, void *y, void *shared_y,
+                                       void *stream);
+
 /* Gate-weighted combine:
  *   out[t,:] = sum_{j<K} topk_w[t,j] * y[inv_perm[t*K+j],:]  (slot order, fp32)
  *            + shared_scale[t] * shared_y[t,:]                (if shared_y != NULL;

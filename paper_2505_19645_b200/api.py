@@ -200,6 +200,29 @@ def moe_grouped_swiglu(cfg, weights, x, grouping: Grouping, y, shared_y, ws, str
         _stream_ptr(stream)), "moe_grouped_swiglu")
 
 
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def moe_grouped_swiglu_static(cfg, weights, x, grouping: Grouping, y, shared_y, stream=None):
+    """moe_grouped_swiglu for callers that cannot hand over a workspace (no allocation may
+    happen where they run, e.g. a server with a frozen memory plan): scratch is a fixed
+    array of STATIC_SCRATCH_BYTES inside the library, shared by all calls on the device.
+    Raises MoeError(MOE_ERR_WORKSPACE) if the request does not fit.  Make the first call on
+    a device outside stream capture; do not let two calls overlap on the GPU."""
+    T = x.shape[0]
+    g = grouping
+    i32 = torch.int32
+    lib = load_library()
+    lib.moe_grouped_swiglu_static.restype = ctypes.c_int32
+    lib.moe_grouped_swiglu_static.argtypes = [
+        ctypes.POINTER(CConfig), ctypes.POINTER(CWeights), ctypes.c_void_p, ctypes.c_int32] + \
+        [ctypes.c_void_p] * 7
+    _check(lib.moe_grouped_swiglu_static(
+        ctypes.byref(cfg), ctypes.byref(weights), _ptr(x, torch.bfloat16), T, _ptr(g.offsets, i32),
+        _ptr(g.perm, i32), _ptr(g.active, i32), _ptr(g.n_active, i32), _ptr(y, torch.bfloat16),
+        _ptr(shared_y, torch.bfloat16), _stream_ptr(stream)), "moe_grouped_swiglu_static")
+
+
 def moe_combine(cfg, y, inv_perm, topk_w, shared_y, shared_scale, out, stream=None):
     T = out.shape[0]
     _check(load_library().moe_combine(

@@ -22,9 +22,9 @@ int sm_count()
 
 static thread_local int g_last_launches = 0;
 
-static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-static moe_status_t check_config(const moe_config_t *c)
+moe_status_t check_config(const moe_config_t *c)
 {
     if (!c)
         return MOE_ERR_INVALID_ARG;
@@ -41,7 +41,7 @@ static moe_status_t check_config(const moe_config_t *c)
     return MOE_OK;
 }
 
-static moe_status_t check_tokens(const moe_config_t *c, int64_t T)
+moe_status_t check_tokens(const moe_config_t *c, int64_t T)
 {
     if (T < 1 || T * c->top_k >= (1 << 24))
         return MOE_ERR_INVALID_ARG;
@@ -49,7 +49,7 @@ static moe_status_t check_tokens(const moe_config_t *c, int64_t T)
 }
 
 // The kernels are built for sm_100a only.
-static moe_status_t check_device()
+moe_status_t check_device()
 {
     static int ok[64];
     int dev = 0;
@@ -66,7 +66,7 @@ static moe_status_t check_device()
     return ok[dev] == 1 ? MOE_OK : MOE_ERR_UNSUPPORTED;
 }
 
-static bool weights_ok(const moe_config_t *c, const moe_weights_t *w, bool need_router,
+bool weights_ok(const moe_config_t *c, const moe_weights_t *w, bool need_router,
                        bool need_experts)
 {
     if (!w)
@@ -117,10 +117,10 @@ static thread_local bool g_probe_armed = false;  // only moe_verify_layer arms i
             return MOE_ERR_CUDA;                                              \
     } while (0)
 
-static moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x,
-                            int T, const int32_t *offsets, const int32_t *perm,
-                            __nv_bfloat16 *y, __nv_bfloat16 *shared_y, char *ws,
-                            const Workspace &L, cudaStream_t s, int &launches)
+moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
+                     const int32_t *offsets, const int32_t *perm, __nv_bfloat16 *y,
+                     __nv_bfloat16 *shared_y, char *ws, const Workspace &L, cudaStream_t s,
+                     int &launches)
 {
     const bool with_shared = shared_y != nullptr && c.shared_inter > 0;
     PlanView plan{reinterpret_cast<int32_t *>(ws + L.plan_header),

@@ -132,6 +132,18 @@ cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, const 
 
 int sm_count();
 
+// Host-side argument checks and the FFN launch sequence shared by the entry points.
+bool aligned16(const void *p);
+moe_status_t check_config(const moe_config_t *c);
+moe_status_t check_tokens(const moe_config_t *c, int64_t T);
+moe_status_t check_device();
+bool weights_ok(const moe_config_t *c, const moe_weights_t *w, bool need_router, bool need_experts);
+// plan -> gate/up + SwiGLU -> down; uses the regions status, plan_*, h, h_shared of `L` in `ws`
+moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
+                     const int32_t *offsets, const int32_t *perm, __nv_bfloat16 *y,
+                     __nv_bfloat16 *shared_y, char *ws, const Workspace &L, cudaStream_t s,
+                     int &launches);
+
 // ---------------------------------------------------------------------------------------
 // Device helpers.
 // ---------------------------------------------------------------------------------------

@@ -1,0 +1,101 @@
+// moe_grouped_swiglu_static: the expert-FFN step for callers that cannot provide scratch.
+//
+// Some users of this library run where device allocation is off the table: a serving
+// loop that fixed its memory plan at start-up and refuses any later cudaMalloc, a plugin
+// inside a host framework that owns the allocator, a real-time path where an allocation
+// could stall on a device-wide synchronisation.  For them the FFN step's scratch (segment
+// plan + SwiGLU intermediates) lives in a fixed array inside the library image itself.
+// The price: every GPU that loads the library carries MOE_STATIC_SCRATCH_BYTES until the
+// process exits, sizes beyond it are refused, and all calls share (and overwrite) it.
+#include <mutex>
+
+#include "common.cuh"
+
+namespace moe {
+
+// The scratch itself.  In host code this name is only a handle for the runtime's symbol
+// table, never a device address: the address comes from cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_static_scratch[MOE_STATIC_SCRATCH_BYTES];
+
+static std::mutex g_scratch_mutex;
+static void *g_scratch_addr[64];  // per device ordinal, resolved on first use
+
+// Device address of the scratch array on the CURRENT device (resolved once per device).
+static moe_status_t static_scratch_address(char **out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    if (dev < 0 || dev >= 64)
+        return MOE_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p)
+            return MOE_ERR_CUDA;
+        g_scratch_addr[dev] = p;
+    }
+    *out = static_cast<char *>(g_scratch_addr[dev]);
+    return MOE_OK;
+}
+
+// Only the regions the FFN step touches, packed from offset 0.
+static Workspace static_scratch_layout(const moe_config_t &c, int T)
+{
+    Workspace w{};
+    const size_t A = (size_t)T * c.top_k;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t at = off;
+        off = align_up(off + bytes, 256);
+        return at;
+    };
+    w.status = take(64 * 4);
+    w.plan_header = take(PLAN_HEADER_INTS * 4);
+    w.plan_routed = take(sizeof(Segment) * (size_t)max_routed_segments(c.n_experts, (int)A));
+    w.plan_shared = take(sizeof(Segment) * (size_t)max_shared_segments(T));
+    w.h = take(A * (size_t)c.inter * 2);
+    w.h_shared = take((size_t)T * c.shared_inter * 2);
+    w.total = off;
+    return w;
+}
+
+}  // namespace moe
+
+using namespace moe;
+
+extern "C" {
+
+moe_status_t moe_grouped_swiglu_static(const moe_config_t *cfg, const moe_weights_t *w,
+                                       const void *x, int32_t T, const int32_t *offsets,
+                                       const int32_t *perm, const int32_t *active,
+                                       const int32_t *n_active, void *y, void *shared_y,
+                                       void *stream)
+{
+    moe_status_t st = check_config(cfg);
+    if (st != MOE_OK)
+        return st;
+    if ((st = check_tokens(cfg, T)) != MOE_OK)
+        return st;
+    if (!weights_ok(cfg, w, false, true) || !x || !offsets || !perm || !active || !n_active || !y)
+        return MOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y) || (shared_y && !aligned16(shared_y)))
+        return MOE_ERR_INVALID_ARG;
+    const Workspace L = static_scratch_layout(*cfg, T);
+    if (L.total > (size_t)MOE_STATIC_SCRATCH_BYTES)
+        return MOE_ERR_WORKSPACE;  // request does not fit the built-in scratch
+    if ((st = check_device()) != MOE_OK)
+        return st;
+    char *scratch = nullptr;
+    if ((st = static_scratch_address(&scratch)) != MOE_OK)
+        return st;
+    int launches = 0;
+    // The plan kernel, first in the sequence, clears the status word and rewrites the whole
+    // plan; h is fully written by the gate/up pass before the down pass reads it.  Nothing
+    // else in the array has to start at zero.
+    return run_ffn(*cfg, *w, static_cast<const __nv_bfloat16 *>(x), T, offsets, perm,
+                   static_cast<__nv_bfloat16 *>(y), static_cast<__nv_bfloat16 *>(shared_y), scratch,
+                   L, static_cast<cudaStream_t>(stream), launches);
+}
+
+}  // extern "C"
