@@ -120,7 +120,7 @@ static thread_local bool g_probe_armed = false;  // only moe_verify_layer arms i
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
                      const int32_t *offsets, const int32_t *perm, __nv_bfloat16 *y,
                      __nv_bfloat16 *shared_y, char *ws, const Workspace &L, cudaStream_t s,
-                     int &launches)
+                     int &launches, bool plan_ready)
 {
     const bool with_shared = shared_y != nullptr && c.shared_inter > 0;
     PlanView plan{reinterpret_cast<int32_t *>(ws + L.plan_header),
@@ -128,8 +128,9 @@ moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_b
                   reinterpret_cast<Segment *>(ws + L.plan_shared)};
     __nv_bfloat16 *h = reinterpret_cast<__nv_bfloat16 *>(ws + L.h);
     __nv_bfloat16 *hs = reinterpret_cast<__nv_bfloat16 *>(ws + L.h_shared);
-    MOE_STAGE(MOE_STAGE_PLAN, launch_plan(c, T, offsets, with_shared,
-                                          reinterpret_cast<int32_t *>(ws + L.status), plan, s));
+    if (!plan_ready)
+        MOE_STAGE(MOE_STAGE_PLAN, launch_plan(c, T, offsets, with_shared,
+                                              reinterpret_cast<int32_t *>(ws + L.status), plan, s));
     MOE_STAGE(MOE_STAGE_GATE_UP,
               launch_ffn_stream_gateup(c, w, x, T, perm, plan, with_shared, h, hs, s));
     MOE_STAGE(MOE_STAGE_DOWN,
@@ -305,9 +306,14 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
     MOE_STAGE(MOE_STAGE_ROUTER_LOGITS,
               launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s));
     MOE_STAGE(MOE_STAGE_ROUTE_TOPK, launch_route_topk(*cfg, logits, T, topk_idx, topk_w, s));
-    MOE_STAGE(MOE_STAGE_PERMUTE, launch_permute(*cfg, topk_idx, T, counts, offsets, perm, inv_perm,
-                                                active, n_active, s));
-    st = run_ffn(*cfg, *w, xb, T, offsets, perm, y, ys, base, L, s, launches);
+    // the grouping kernel also writes the FFN segment plan (one launch fewer)
+    const PlanView plan{reinterpret_cast<int32_t *>(base + L.plan_header),
+                        reinterpret_cast<Segment *>(base + L.plan_routed),
+                        reinterpret_cast<Segment *>(base + L.plan_shared)};
+    MOE_STAGE(MOE_STAGE_PERMUTE,
+              launch_permute(*cfg, topk_idx, T, counts, offsets, perm, inv_perm, active, n_active, s,
+                             &plan, has_shared, reinterpret_cast<int32_t *>(base + L.status)));
+    st = run_ffn(*cfg, *w, xb, T, offsets, perm, y, ys, base, L, s, launches, true);
     if (st != MOE_OK)
         return st;
     MOE_STAGE(MOE_STAGE_COMBINE,

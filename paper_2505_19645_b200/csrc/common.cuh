@@ -113,7 +113,8 @@ cudaError_t launch_route_topk(const moe_config_t &c, const float *logits, int T,
                               float *wts, cudaStream_t s);
 cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int32_t *counts,
                            int32_t *offsets, int32_t *perm, int32_t *inv_perm, int32_t *active,
-                           int32_t *n_active, cudaStream_t s);
+                           int32_t *n_active, cudaStream_t s, const PlanView *plan = nullptr,
+                           bool with_shared = false, int32_t *status = nullptr);
 cudaError_t launch_plan(const moe_config_t &c, int T, const int32_t *offsets, bool with_shared,
                         int32_t *status, PlanView plan, cudaStream_t s);
 // gate/up + SwiGLU for every segment of the plan: h[row,:] (routed) and h_shared[row,:]
@@ -142,7 +143,7 @@ bool weights_ok(const moe_config_t *c, const moe_weights_t *w, bool need_router,
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
                      const int32_t *offsets, const int32_t *perm, __nv_bfloat16 *y,
                      __nv_bfloat16 *shared_y, char *ws, const Workspace &L, cudaStream_t s,
-                     int &launches);
+                     int &launches, bool plan_ready = false);
 
 // ---------------------------------------------------------------------------------------
 // Device helpers.

@@ -39,7 +39,9 @@ __global__ void __launch_bounds__(PERM_THREADS)
 permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__restrict__ counts,
                int32_t *__restrict__ offsets, int32_t *__restrict__ perm,
                int32_t *__restrict__ inv_perm, int32_t *__restrict__ active,
-               int32_t *__restrict__ n_active)
+               int32_t *__restrict__ n_active, int T, int with_shared,
+               int32_t *__restrict__ status, int32_t *__restrict__ plan_header,
+               Segment *__restrict__ plan_routed, Segment *__restrict__ plan_shared)
 {
     __shared__ int hist[MOE_MAX_EXPERTS];
     __shared__ int offs[MOE_MAX_EXPERTS];
@@ -79,6 +81,42 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
             active[tid] = -1;
         if (tid == 0)
             n_active[0] = total;
+        // Inside moe_verify_layer the segment plan of the FFN kernels is written here as
+        // well (same content as plan_kernel), which saves a launch.
+        if (plan_header != nullptr) {
+            __syncthreads();
+            const int cnt = tid < E ? hist[tid] : 0;
+            if (tid < MOE_MAX_EXPERTS)
+                flag[tid] = (cnt + SEG_TOKENS - 1) / SEG_TOKENS;
+            __syncthreads();
+            block_exclusive_scan(flag, tmp, E, &total);
+            if (tid < E) {
+                int at = flag[tid];
+                const int row0 = offs[tid];
+                for (int r = 0; r < cnt; r += SEG_TOKENS) {
+                    Segment sg;
+                    sg.expert = tid;
+                    sg.row0 = row0 + r;
+                    sg.n = min(SEG_TOKENS, cnt - r);
+                    sg.pad = 0;
+                    plan_routed[at++] = sg;
+                }
+            }
+            const int n_shared = with_shared ? (T + SEG_TOKENS - 1) / SEG_TOKENS : 0;
+            for (int i = tid; i < n_shared; i += PERM_THREADS) {
+                Segment sg;
+                sg.expert = -1;
+                sg.row0 = i * SEG_TOKENS;
+                sg.n = min(SEG_TOKENS, T - i * SEG_TOKENS);
+                sg.pad = 0;
+                plan_shared[i] = sg;
+            }
+            if (tid == 0) {
+                plan_header[0] = total;
+                plan_header[1] = n_shared;
+                status[0] = 0;
+            }
+        }
     }
 
     const int warp = tid >> 5, lane = tid & 31;
@@ -111,12 +149,15 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
 
 cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int32_t *counts,
                            int32_t *offsets, int32_t *perm, int32_t *inv_perm, int32_t *active,
-                           int32_t *n_active, cudaStream_t s)
+                           int32_t *n_active, cudaStream_t s, const PlanView *plan,
+                           bool with_shared, int32_t *status)
 {
     const int E = c.n_experts;
     const int blocks = (E + 31) / 32;
-    permute_kernel<<<blocks, PERM_THREADS, 0, s>>>(idx, T * c.top_k, E, counts, offsets, perm,
-                                                   inv_perm, active, n_active);
+    permute_kernel<<<blocks, PERM_THREADS, 0, s>>>(
+        idx, T * c.top_k, E, counts, offsets, perm, inv_perm, active, n_active, T,
+        with_shared ? 1 : 0, status, plan ? plan->header : nullptr, plan ? plan->routed : nullptr,
+        plan ? plan->shared : nullptr);
     return cudaGetLastError();
 }
 

@@ -1,0 +1,176 @@
+// Router logits  z[t,e] = x[t,:] . w_router[e,:] (+ bias[e])  and the shared expert's scalar
+// gate  s[t] = sigmoid(x[t,:] . w_sg), with fp32-level accuracy on the tensor cores.
+//
+// The fp32 router row is split on the fly into three bf16 terms  w = hi + mid + lo  (each
+// remainder is exact in fp32, so the three terms carry 24 mantissa bits), the bf16 token
+// values are exact, and the three partial products are accumulated in fp32 by
+// m16n8k16 MMAs.  A CTA owns 16 router rows x (8*NCH) tokens; its 8 warps split H and are
+// summed through shared memory, so even T = 1 keeps every load short and parallel.
+#include "common.cuh"
+
+namespace moe {
+
+constexpr int RL_WARPS = 8;
+
+struct Split3 {
+    uint32_t hi, mid, lo;  // two bf16 each
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b)
+{
+    __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&p);
+}
+
+__device__ __forceinline__ Split3 split_pair(float a, float b)
+{
+    Split3 s;
+    s.hi = pack_bf16x2(a, b);
+    const float ra = a - bf16_lo(s.hi), rb = b - bf16_hi(s.hi);
+    s.mid = pack_bf16x2(ra, rb);
+    const float ra2 = ra - bf16_lo(s.mid), rb2 = rb - bf16_hi(s.mid);
+    s.lo = pack_bf16x2(ra2, rb2);
+    return s;
+}
+
+// 8 consecutive values of one router row as fp32 (row kinds: fp32 router row, the bf16
+// shared-gate vector, or a padding row of zeros).
+struct RowSrc {
+    const float *f32;           // non-null: fp32 row
+    const __nv_bfloat16 *bf16;  // non-null: bf16 row
+};
+
+__device__ __forceinline__ void load_row8(const RowSrc &r, int k, float (&v)[8])
+{
+    if (r.f32) {
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(r.f32 + k));
+        const float4 b = __ldg(reinterpret_cast<const float4 *>(r.f32 + k + 4));
+        v[0] = a.x, v[1] = a.y, v[2] = a.z, v[3] = a.w;
+        v[4] = b.x, v[5] = b.y, v[6] = b.z, v[7] = b.w;
+    } else if (r.bf16) {
+        const uint4 p = __ldg(reinterpret_cast<const uint4 *>(r.bf16 + k));
+        v[0] = bf16_lo(p.x), v[1] = bf16_hi(p.x), v[2] = bf16_lo(p.y), v[3] = bf16_hi(p.y);
+        v[4] = bf16_lo(p.z), v[5] = bf16_hi(p.z), v[6] = bf16_lo(p.w), v[7] = bf16_hi(p.w);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            v[i] = 0.f;
+    }
+}
+
+template <int NCH>
+__global__ void __launch_bounds__(RL_WARPS * 32)
+router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ w_router,
+                     const float *__restrict__ bias, const __nv_bfloat16 *__restrict__ w_sg,
+                     int T, int H, int E, int n_rows, float *__restrict__ logits,
+                     float *__restrict__ shared_scale)
+{
+    __shared__ float part[RL_WARPS][NCH][4][32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;
+    const int e0 = blockIdx.x * 16;
+    const int t0 = blockIdx.y * (8 * NCH);
+
+    auto row_src = [&](int e) {
+        RowSrc r{nullptr, nullptr};
+        if (e < E)
+            r.f32 = w_router + (size_t)e * H + 8 * tq;
+        else if (e == E && e < n_rows)
+            r.bf16 = w_sg + 8 * tq;
+        return r;
+    };
+    const RowSrc rlo = row_src(e0 + g), rhi = row_src(e0 + g + 8);
+    const __nv_bfloat16 *b[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c)
+        b[c] = x + (size_t)min(t0 + c * 8 + g, T - 1) * H + 8 * tq;
+
+    float acc[NCH][4];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c)
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            acc[c][q] = 0.f;
+
+    const int nsteps = H >> 5;
+    const int s0 = warp * nsteps / RL_WARPS, s1 = (warp + 1) * nsteps / RL_WARPS;
+#pragma unroll 2
+    for (int s = s0; s < s1; ++s) {
+        const int k = s * 32;
+        float lo8[8], hi8[8];
+        load_row8(rlo, k, lo8);
+        load_row8(rhi, k, hi8);
+        uint4 B[NCH];
+#pragma unroll
+        for (int c = 0; c < NCH; ++c)
+            B[c] = ld_cached_v4(b[c] + k);
+        // physical k positions 8tq+{0..3} feed the first MMA, 8tq+{4..7} the second
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const Split3 a0 = split_pair(lo8[4 * half + 0], lo8[4 * half + 1]);
+            const Split3 a1 = split_pair(hi8[4 * half + 0], hi8[4 * half + 1]);
+            const Split3 a2 = split_pair(lo8[4 * half + 2], lo8[4 * half + 3]);
+            const Split3 a3 = split_pair(hi8[4 * half + 2], hi8[4 * half + 3]);
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                const uint32_t b0 = half ? B[c].z : B[c].x, b1 = half ? B[c].w : B[c].y;
+                mma_bf16_16816(acc[c], a0.lo, a1.lo, a2.lo, a3.lo, b0, b1);
+                mma_bf16_16816(acc[c], a0.mid, a1.mid, a2.mid, a3.mid, b0, b1);
+                mma_bf16_16816(acc[c], a0.hi, a1.hi, a2.hi, a3.hi, b0, b1);
+            }
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < NCH; ++c)
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            part[warp][c][q][lane] = acc[c][q];
+    __syncthreads();
+
+    // accumulator q of lane (g,tq), chunk c: row g + 8*(q>>1), token c*8 + 2*tq + (q&1)
+    for (int o = threadIdx.x; o < 16 * 8 * NCH; o += RL_WARPS * 32) {
+        const int r = o & 15, slot = o >> 4;
+        const int c = slot >> 3, tt = (slot & 7) >> 1, lo = slot & 1;
+        const int q = ((r >> 3) << 1) | lo, ln = ((r & 7) << 2) | tt;
+        const int e = e0 + r, t = t0 + slot;
+        if (e >= n_rows || t >= T)
+            continue;
+        float v = 0.f;
+#pragma unroll
+        for (int w = 0; w < RL_WARPS; ++w)
+            v += part[w][c][q][ln];
+        if (e < E)
+            logits[(size_t)t * E + e] = bias ? v + bias[e] : v;
+        else
+            shared_scale[t] = 1.0f / (1.0f + expf(-v));
+    }
+}
+
+cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
+                                 const __nv_bfloat16 *x, int T, float *logits,
+                                 float *shared_scale, cudaStream_t s)
+{
+    const bool gate_row = shared_scale != nullptr && c.shared_gate && c.shared_inter > 0;
+    const int n_rows = c.n_experts + (gate_row ? 1 : 0);
+    const int e_tiles = (n_rows + 15) / 16;
+    // the smallest token tile that keeps the grid within about two waves
+    int nch = 1;
+    while (nch < 8 && (long long)e_tiles * ((T + 8 * nch - 1) / (8 * nch)) > 2LL * sm_count())
+        nch *= 2;
+    dim3 grid(e_tiles, (T + 8 * nch - 1) / (8 * nch));
+    const __nv_bfloat16 *w_sg = static_cast<const __nv_bfloat16 *>(w.w_shared_gate);
+#define MOE_RL_LAUNCH(N)                                                                    \
+    router_logits_kernel<N><<<grid, RL_WARPS * 32, 0, s>>>(x, w.w_router, w.router_bias, w_sg, T, \
+                                                          c.hidden, c.n_experts, n_rows, logits, \
+                                                          shared_scale)
+    switch (nch) {
+    case 1: MOE_RL_LAUNCH(1); break;
+    case 2: MOE_RL_LAUNCH(2); break;
+    case 4: MOE_RL_LAUNCH(4); break;
+    default: MOE_RL_LAUNCH(8); break;
+    }
+#undef MOE_RL_LAUNCH
+    return cudaGetLastError();
+}
+
+}  // namespace moe
