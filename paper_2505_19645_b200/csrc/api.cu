@@ -117,24 +117,44 @@ static thread_local bool g_probe_armed = false;  // only moe_verify_layer arms i
             return MOE_ERR_CUDA;                                              \
     } while (0)
 
+PlanView plan_view(char *ws, const Workspace &L)
+{
+    return PlanView{reinterpret_cast<int32_t *>(ws + L.plan_header),
+                    reinterpret_cast<Segment *>(ws + L.plan_routed),
+                    reinterpret_cast<Segment *>(ws + L.plan_shared),
+                    reinterpret_cast<Segment *>(ws + L.plan_tc_routed),
+                    reinterpret_cast<Segment *>(ws + L.plan_tc_shared)};
+}
+
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
                      const int32_t *offsets, const int32_t *perm, __nv_bfloat16 *y,
                      __nv_bfloat16 *shared_y, char *ws, const Workspace &L, cudaStream_t s,
                      int &launches, bool plan_ready)
 {
     const bool with_shared = shared_y != nullptr && c.shared_inter > 0;
-    PlanView plan{reinterpret_cast<int32_t *>(ws + L.plan_header),
-                  reinterpret_cast<Segment *>(ws + L.plan_routed),
-                  reinterpret_cast<Segment *>(ws + L.plan_shared)};
+    const PlanView plan = plan_view(ws, L);
+    int32_t *status = reinterpret_cast<int32_t *>(ws + L.status);
     __nv_bfloat16 *h = reinterpret_cast<__nv_bfloat16 *>(ws + L.h);
     __nv_bfloat16 *hs = reinterpret_cast<__nv_bfloat16 *>(ws + L.h_shared);
+    __nv_bfloat16 *xs = reinterpret_cast<__nv_bfloat16 *>(ws + L.x_sorted);
+    // no group can have more than T rows: below the threshold the tensor-core kernels have
+    // nothing to do and are not launched at all
+    const bool tc = T > TC_MIN_ROWS;
     if (!plan_ready)
-        MOE_STAGE(MOE_STAGE_PLAN, launch_plan(c, T, offsets, with_shared,
-                                              reinterpret_cast<int32_t *>(ws + L.status), plan, s));
+        MOE_STAGE(MOE_STAGE_PLAN,
+                  launch_plan(c, T, offsets, with_shared, TC_MIN_ROWS, status, plan, s));
+    if (tc)
+        MOE_STAGE(MOE_STAGE_GATHER, launch_gather_rows(c, x, perm, T, xs, s));
     MOE_STAGE(MOE_STAGE_GATE_UP,
               launch_ffn_stream_gateup(c, w, x, T, perm, plan, with_shared, h, hs, s));
+    if (tc)
+        MOE_STAGE(MOE_STAGE_GATE_UP_TC,
+                  launch_ffn_tc_gateup(c, w, x, xs, T, plan, with_shared, h, hs, status, s));
     MOE_STAGE(MOE_STAGE_DOWN,
               launch_ffn_stream_down(c, w, T, plan, with_shared, h, hs, y, shared_y, s));
+    if (tc)
+        MOE_STAGE(MOE_STAGE_DOWN_TC,
+                  launch_ffn_tc_down(c, w, T, plan, with_shared, h, hs, y, shared_y, status, s));
     return MOE_OK;
 }
 
@@ -307,12 +327,11 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
               launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s));
     MOE_STAGE(MOE_STAGE_ROUTE_TOPK, launch_route_topk(*cfg, logits, T, topk_idx, topk_w, s));
     // the grouping kernel also writes the FFN segment plan (one launch fewer)
-    const PlanView plan{reinterpret_cast<int32_t *>(base + L.plan_header),
-                        reinterpret_cast<Segment *>(base + L.plan_routed),
-                        reinterpret_cast<Segment *>(base + L.plan_shared)};
+    const PlanView plan = plan_view(base, L);
     MOE_STAGE(MOE_STAGE_PERMUTE,
               launch_permute(*cfg, topk_idx, T, counts, offsets, perm, inv_perm, active, n_active, s,
-                             &plan, has_shared, reinterpret_cast<int32_t *>(base + L.status)));
+                             &plan, has_shared, TC_MIN_ROWS,
+                             reinterpret_cast<int32_t *>(base + L.status)));
     st = run_ffn(*cfg, *w, xb, T, offsets, perm, y, ys, base, L, s, launches, true);
     if (st != MOE_OK)
         return st;
@@ -356,7 +375,7 @@ moe_status_t moe_check(void *ws, void *stream)
 
 moe_status_t moe_profile_stage(int32_t stage, void *start_event, void *stop_event)
 {
-    if (stage > MOE_STAGE_COMBINE || (stage >= 0 && (!start_event || !stop_event)))
+    if (stage > MOE_STAGE_DOWN_TC || (stage >= 0 && (!start_event || !stop_event)))
         return MOE_ERR_INVALID_ARG;
     g_probe.stage = stage < 0 ? -1 : stage;
     g_probe.start = static_cast<cudaEvent_t>(start_event);

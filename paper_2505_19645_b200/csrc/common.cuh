@@ -14,7 +14,9 @@ namespace moe {
 // plan kernel derives the list from the grouping offsets on the device, so the host never
 // needs the data-dependent counts and no launch waits for a copy.
 // ---------------------------------------------------------------------------------------
-constexpr int SEG_TOKENS = 32;   // rows per segment of the streaming path (4 MMA n-chunks)
+constexpr int SEG_TOKENS = 32;      // rows per segment of the streaming path (4 MMA n-chunks)
+constexpr int TC_SEG_TOKENS = 128;  // rows per segment of the tensor-core path (UMMA N)
+constexpr int TC_MIN_ROWS = 32;     // groups with more rows than this take the tensor-core path
 constexpr int PLAN_HEADER_INTS = 16;
 
 struct Segment {
@@ -24,11 +26,14 @@ struct Segment {
     int32_t pad;
 };
 
-// plan header (ints): [0] routed segments, [1] shared segments
+// plan header (ints): [0] routed / [1] shared streaming segments,
+//                     [2] routed / [3] shared tensor-core segments
 struct PlanView {
     int32_t *header;
-    Segment *routed;  // capacity max_routed_segments()
-    Segment *shared;  // capacity max_shared_segments()
+    Segment *routed;     // capacity max_routed_segments()
+    Segment *shared;     // capacity max_shared_segments()
+    Segment *tc_routed;  // capacity max_tc_routed_segments()
+    Segment *tc_shared;  // capacity max_tc_shared_segments()
 };
 
 __host__ __device__ inline int max_routed_segments(int E, int A)
@@ -38,6 +43,14 @@ __host__ __device__ inline int max_routed_segments(int E, int A)
 __host__ __device__ inline int max_shared_segments(int T)
 {
     return (T + SEG_TOKENS - 1) / SEG_TOKENS;
+}
+__host__ __device__ inline int max_tc_routed_segments(int E, int A)
+{
+    return E + A / TC_SEG_TOKENS + 1;
+}
+__host__ __device__ inline int max_tc_shared_segments(int T)
+{
+    return (T + TC_SEG_TOKENS - 1) / TC_SEG_TOKENS;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -58,6 +71,9 @@ struct Workspace {
     size_t plan_header;   // i32 [PLAN_HEADER_INTS]
     size_t plan_routed;   // Segment[max_routed_segments]
     size_t plan_shared;   // Segment[max_shared_segments]
+    size_t plan_tc_routed;  // Segment[max_tc_routed_segments]
+    size_t plan_tc_shared;  // Segment[max_tc_shared_segments]
+    size_t x_sorted;      // bf16 [A, H]      token rows in sorted order (tensor-core path)
     size_t h;             // bf16 [A, I]      SwiGLU intermediate, sorted order
     size_t h_shared;      // bf16 [T, I_s]
     size_t y;             // bf16 [A, H]      expert outputs, sorted order
@@ -91,6 +107,9 @@ inline Workspace workspace_layout(const moe_config_t &c, int T)
     w.plan_header = take(PLAN_HEADER_INTS * 4);
     w.plan_routed = take(sizeof(Segment) * (size_t)max_routed_segments((int)E, (int)A));
     w.plan_shared = take(sizeof(Segment) * (size_t)max_shared_segments(T));
+    w.plan_tc_routed = take(sizeof(Segment) * (size_t)max_tc_routed_segments((int)E, (int)A));
+    w.plan_tc_shared = take(sizeof(Segment) * (size_t)max_tc_shared_segments(T));
+    w.x_sorted = take(T > TC_MIN_ROWS ? A * H * 2 : 0);
     w.h = take(A * (size_t)c.inter * 2);
     w.h_shared = take((size_t)T * c.shared_inter * 2);
     w.y = take(A * H * 2);
@@ -114,9 +133,21 @@ cudaError_t launch_route_topk(const moe_config_t &c, const float *logits, int T,
 cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int32_t *counts,
                            int32_t *offsets, int32_t *perm, int32_t *inv_perm, int32_t *active,
                            int32_t *n_active, cudaStream_t s, const PlanView *plan = nullptr,
-                           bool with_shared = false, int32_t *status = nullptr);
+                           bool with_shared = false, int tc_min_rows = TC_MIN_ROWS,
+                           int32_t *status = nullptr);
 cudaError_t launch_plan(const moe_config_t &c, int T, const int32_t *offsets, bool with_shared,
-                        int32_t *status, PlanView plan, cudaStream_t s);
+                        int tc_min_rows, int32_t *status, PlanView plan, cudaStream_t s);
+// tensor-core path (groups with more than TC_MIN_ROWS rows)
+cudaError_t launch_gather_rows(const moe_config_t &c, const __nv_bfloat16 *x, const int32_t *perm,
+                               int T, __nv_bfloat16 *x_sorted, cudaStream_t s);
+cudaError_t launch_ffn_tc_gateup(const moe_config_t &c, const moe_weights_t &w,
+                                 const __nv_bfloat16 *x, const __nv_bfloat16 *x_sorted, int T,
+                                 PlanView plan, bool with_shared, __nv_bfloat16 *h,
+                                 __nv_bfloat16 *h_shared, int32_t *status, cudaStream_t s);
+cudaError_t launch_ffn_tc_down(const moe_config_t &c, const moe_weights_t &w, int T, PlanView plan,
+                               bool with_shared, const __nv_bfloat16 *h,
+                               const __nv_bfloat16 *h_shared, __nv_bfloat16 *y,
+                               __nv_bfloat16 *y_shared, int32_t *status, cudaStream_t s);
 // gate/up + SwiGLU for every segment of the plan: h[row,:] (routed) and h_shared[row,:]
 cudaError_t launch_ffn_stream_gateup(const moe_config_t &c, const moe_weights_t &w,
                                      const __nv_bfloat16 *x, int T, const int32_t *perm,
@@ -139,6 +170,7 @@ moe_status_t check_config(const moe_config_t *c);
 moe_status_t check_tokens(const moe_config_t *c, int64_t T);
 moe_status_t check_device();
 bool weights_ok(const moe_config_t *c, const moe_weights_t *w, bool need_router, bool need_experts);
+PlanView plan_view(char *ws, const Workspace &L);
 // plan -> gate/up + SwiGLU -> down; uses the regions status, plan_*, h, h_shared of `L` in `ws`
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
                      const int32_t *offsets, const int32_t *perm, __nv_bfloat16 *y,

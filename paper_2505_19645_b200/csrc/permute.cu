@@ -31,17 +31,71 @@ __device__ void block_exclusive_scan(int *vals, int *tmp, int n, int *total)
     __syncthreads();
 }
 
+// Segment plan from per-expert counts and offsets held in shared memory.  A group (expert, or
+// the shared expert with its T rows) with at most tc_min_rows rows is cut into streaming
+// segments of <= SEG_TOKENS rows; a larger group into tensor-core segments of <= TC_SEG_TOKENS
+// rows.  All threads of the block must call it; scan/tmp/total are shared scratch.
+__device__ void build_plan(const int *cnt_sh, const int *off_sh, int *scan, int *tmp, int *total,
+                           int E, int T, int with_shared, int tc_min_rows, int32_t *status,
+                           PlanView plan)
+{
+    const int tid = threadIdx.x;
+    const int cnt = tid < E ? cnt_sh[tid] : 0;
+    const int row0 = tid < E ? off_sh[tid] : 0;
+    const bool tc = cnt > tc_min_rows;
+    for (int pass = 0; pass < 2; ++pass) {
+        const int seg_rows = pass == 0 ? SEG_TOKENS : TC_SEG_TOKENS;
+        const bool mine = cnt > 0 && (pass == 0 ? !tc : tc);
+        __syncthreads();
+        if (tid < MOE_MAX_EXPERTS)
+            scan[tid] = mine ? (cnt + seg_rows - 1) / seg_rows : 0;
+        __syncthreads();
+        block_exclusive_scan(scan, tmp, E, total);
+        Segment *list = pass == 0 ? plan.routed : plan.tc_routed;
+        if (mine) {
+            int at = scan[tid];
+            for (int r = 0; r < cnt; r += seg_rows) {
+                Segment sg;
+                sg.expert = tid;
+                sg.row0 = row0 + r;
+                sg.n = min(seg_rows, cnt - r);
+                sg.pad = 0;
+                list[at++] = sg;
+            }
+        }
+        if (tid == 0)
+            plan.header[pass == 0 ? 0 : 2] = *total;
+    }
+    const bool shared_tc = T > tc_min_rows;
+    const int seg_rows = shared_tc ? TC_SEG_TOKENS : SEG_TOKENS;
+    const int n_shared = with_shared ? (T + seg_rows - 1) / seg_rows : 0;
+    Segment *slist = shared_tc ? plan.tc_shared : plan.shared;
+    for (int i = tid; i < n_shared; i += blockDim.x) {
+        Segment sg;
+        sg.expert = -1;
+        sg.row0 = i * seg_rows;
+        sg.n = min(seg_rows, T - i * seg_rows);
+        sg.pad = 0;
+        slist[i] = sg;
+    }
+    if (tid == 0) {
+        plan.header[1] = shared_tc ? 0 : n_shared;
+        plan.header[3] = shared_tc ? n_shared : 0;
+        status[0] = 0;  // device status word: cleared at the start of every FFN pass
+    }
+}
+
 // Every CTA rebuilds the (tiny) histogram and scan for itself, so no grid-wide
 // dependency is needed; CTA b then places experts 32b .. 32b+31, one warp each, walking
 // the assignments in ascending order (ballot + prefix popcount) -- stable by construction,
-// no atomics decide a position.  CTA 0 also writes counts / offsets / active / n_active.
+// no atomics decide a position.  CTA 0 also writes counts / offsets / active / n_active and,
+// inside moe_verify_layer, the FFN segment plan (one launch fewer).
 __global__ void __launch_bounds__(PERM_THREADS)
 permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__restrict__ counts,
                int32_t *__restrict__ offsets, int32_t *__restrict__ perm,
                int32_t *__restrict__ inv_perm, int32_t *__restrict__ active,
-               int32_t *__restrict__ n_active, int T, int with_shared,
-               int32_t *__restrict__ status, int32_t *__restrict__ plan_header,
-               Segment *__restrict__ plan_routed, Segment *__restrict__ plan_shared)
+               int32_t *__restrict__ n_active, int T, int with_shared, int tc_min_rows,
+               int32_t *__restrict__ status, PlanView plan)
 {
     __shared__ int hist[MOE_MAX_EXPERTS];
     __shared__ int offs[MOE_MAX_EXPERTS];
@@ -81,42 +135,8 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
             active[tid] = -1;
         if (tid == 0)
             n_active[0] = total;
-        // Inside moe_verify_layer the segment plan of the FFN kernels is written here as
-        // well (same content as plan_kernel), which saves a launch.
-        if (plan_header != nullptr) {
-            __syncthreads();
-            const int cnt = tid < E ? hist[tid] : 0;
-            if (tid < MOE_MAX_EXPERTS)
-                flag[tid] = (cnt + SEG_TOKENS - 1) / SEG_TOKENS;
-            __syncthreads();
-            block_exclusive_scan(flag, tmp, E, &total);
-            if (tid < E) {
-                int at = flag[tid];
-                const int row0 = offs[tid];
-                for (int r = 0; r < cnt; r += SEG_TOKENS) {
-                    Segment sg;
-                    sg.expert = tid;
-                    sg.row0 = row0 + r;
-                    sg.n = min(SEG_TOKENS, cnt - r);
-                    sg.pad = 0;
-                    plan_routed[at++] = sg;
-                }
-            }
-            const int n_shared = with_shared ? (T + SEG_TOKENS - 1) / SEG_TOKENS : 0;
-            for (int i = tid; i < n_shared; i += PERM_THREADS) {
-                Segment sg;
-                sg.expert = -1;
-                sg.row0 = i * SEG_TOKENS;
-                sg.n = min(SEG_TOKENS, T - i * SEG_TOKENS);
-                sg.pad = 0;
-                plan_shared[i] = sg;
-            }
-            if (tid == 0) {
-                plan_header[0] = total;
-                plan_header[1] = n_shared;
-                status[0] = 0;
-            }
-        }
+        if (plan.header != nullptr)
+            build_plan(hist, offs, flag, tmp, &total, E, T, with_shared, tc_min_rows, status, plan);
     }
 
     const int warp = tid >> 5, lane = tid & 31;
@@ -150,69 +170,46 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
 cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int32_t *counts,
                            int32_t *offsets, int32_t *perm, int32_t *inv_perm, int32_t *active,
                            int32_t *n_active, cudaStream_t s, const PlanView *plan,
-                           bool with_shared, int32_t *status)
+                           bool with_shared, int tc_min_rows, int32_t *status)
 {
     const int E = c.n_experts;
     const int blocks = (E + 31) / 32;
-    permute_kernel<<<blocks, PERM_THREADS, 0, s>>>(
-        idx, T * c.top_k, E, counts, offsets, perm, inv_perm, active, n_active, T,
-        with_shared ? 1 : 0, status, plan ? plan->header : nullptr, plan ? plan->routed : nullptr,
-        plan ? plan->shared : nullptr);
+    PlanView pv{};
+    if (plan)
+        pv = *plan;
+    permute_kernel<<<blocks, PERM_THREADS, 0, s>>>(idx, T * c.top_k, E, counts, offsets, perm,
+                                                   inv_perm, active, n_active, T,
+                                                   with_shared ? 1 : 0, tc_min_rows, status, pv);
     return cudaGetLastError();
 }
 
-// ---------------------------------------------------------------------------------------
-// Segment plan: cut every expert's run of sorted rows into segments of <= SEG_TOKENS rows.
-// ---------------------------------------------------------------------------------------
+// Stand-alone plan (moe_grouped_swiglu gets its offsets from the caller).
 __global__ void __launch_bounds__(MOE_MAX_EXPERTS)
-plan_kernel(const int32_t *__restrict__ offsets, int E, int T, int with_shared,
-            int32_t *__restrict__ status, int32_t *__restrict__ header,
-            Segment *__restrict__ routed, Segment *__restrict__ shared)
+plan_kernel(const int32_t *__restrict__ offsets, int E, int T, int with_shared, int tc_min_rows,
+            int32_t *__restrict__ status, PlanView plan)
 {
-    __shared__ int nseg[MOE_MAX_EXPERTS];
+    __shared__ int cnt[MOE_MAX_EXPERTS];
+    __shared__ int offs[MOE_MAX_EXPERTS];
+    __shared__ int scan[MOE_MAX_EXPERTS];
     __shared__ int tmp[MOE_MAX_EXPERTS];
     __shared__ int total;
     const int tid = threadIdx.x;
-    int row0 = 0, cnt = 0;
+    int row0 = 0, n = 0;
     if (tid < E) {
         row0 = offsets[tid];
-        cnt = offsets[tid + 1] - row0;
+        n = offsets[tid + 1] - row0;
     }
-    nseg[tid] = (cnt + SEG_TOKENS - 1) / SEG_TOKENS;
+    cnt[tid] = n;
+    offs[tid] = row0;
     __syncthreads();
-    block_exclusive_scan(nseg, tmp, E, &total);
-    if (tid < E) {
-        int at = nseg[tid];
-        for (int r = 0; r < cnt; r += SEG_TOKENS) {
-            Segment sg;
-            sg.expert = tid;
-            sg.row0 = row0 + r;
-            sg.n = min(SEG_TOKENS, cnt - r);
-            sg.pad = 0;
-            routed[at++] = sg;
-        }
-    }
-    const int n_shared = with_shared ? (T + SEG_TOKENS - 1) / SEG_TOKENS : 0;
-    for (int i = tid; i < n_shared; i += blockDim.x) {
-        Segment sg;
-        sg.expert = -1;
-        sg.row0 = i * SEG_TOKENS;
-        sg.n = min(SEG_TOKENS, T - i * SEG_TOKENS);
-        sg.pad = 0;
-        shared[i] = sg;
-    }
-    if (tid == 0) {
-        header[0] = total;
-        header[1] = n_shared;
-        status[0] = 0;  // device status word: cleared at the start of every FFN pass
-    }
+    build_plan(cnt, offs, scan, tmp, &total, E, T, with_shared, tc_min_rows, status, plan);
 }
 
 cudaError_t launch_plan(const moe_config_t &c, int T, const int32_t *offsets, bool with_shared,
-                        int32_t *status, PlanView plan, cudaStream_t s)
+                        int tc_min_rows, int32_t *status, PlanView plan, cudaStream_t s)
 {
-    plan_kernel<<<1, MOE_MAX_EXPERTS, 0, s>>>(offsets, c.n_experts, T, with_shared ? 1 : 0, status,
-                                              plan.header, plan.routed, plan.shared);
+    plan_kernel<<<1, MOE_MAX_EXPERTS, 0, s>>>(offsets, c.n_experts, T, with_shared ? 1 : 0,
+                                              tc_min_rows, status, plan);
     return cudaGetLastError();
 }
 
