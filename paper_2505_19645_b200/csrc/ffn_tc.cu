@@ -380,6 +380,7 @@ ffn_tc_kernel(const TcArgs args, const __grid_constant__ CUtensorMap map_a0_r,
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
+        __syncwarp();  // lane 0 arrived from the issue loop: reconverge for the aligned dealloc
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                      "r"(TC_TMEM_COLS)
