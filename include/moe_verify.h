@@ -146,8 +146,7 @@ moe_status_t moe_grouped_swiglu(const moe_config_t *cfg, const moe_weights_t *w,
  * until the process exits.  The call itself allocates nothing, on host or device.
  *
  * Limit: the request must satisfy, with A = T*top_k and every term rounded up to 256 bytes,
- *   256 + 64 + 16*(n_experts + A/32 + 1) + 16*ceil(T/32) + 16*(n_experts + A/128 + 1)
- *     + 16*ceil(T/128) + 2*A*inter + 2*T*shared_inter + (T > 32 ? 2*A*hidden : 0)
+ *   256 + 64 + 16*(n_experts + A/128 + 1) + 2*A*hidden + 2*A*inter + 2*T*shared_inter
  *     <= MOE_STATIC_SCRATCH_BYTES,
  * otherwise MOE_ERR_WORKSPACE is returned and nothing is launched (use moe_grouped_swiglu).
  *
@@ -201,9 +200,7 @@ typedef enum {
     MOE_STAGE_GATE_UP = 4,
     MOE_STAGE_DOWN = 5,
     MOE_STAGE_COMBINE = 6,
-    MOE_STAGE_GATHER = 7,     /* token rows into sorted order (tensor-core path only) */
-    MOE_STAGE_GATE_UP_TC = 8, /* gate/up + SwiGLU of the groups on the tensor-core path */
-    MOE_STAGE_DOWN_TC = 9     /* down projection of the groups on the tensor-core path */
+    MOE_STAGE_GATHER = 7 /* token rows into sorted order */
 } moe_stage_t;
 moe_status_t moe_profile_stage(int32_t stage, void *start_event, void *stop_event);
 

@@ -24,7 +24,7 @@ EXPORTS = ["moe_workspace_bytes", "moe_router_logits", "moe_route_topk", "moe_pe
            "moe_last_launch_count", "moe_status_string", "moe_profile_stage"]
 
 STAGES = {"router_logits": 0, "route_topk": 1, "permute": 2, "plan": 3, "gate_up": 4, "down": 5,
-          "combine": 6, "gather": 7, "gate_up_tc": 8, "down_tc": 9}
+          "combine": 6, "gather": 7}
 
 
 class MoeError(RuntimeError):

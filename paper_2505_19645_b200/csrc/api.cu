@@ -1,4 +1,6 @@
 // C ABI: argument validation, workspace carving and launch sequencing.  No compute here.
+#include <stdlib.h>
+
 #include <mutex>
 
 #include "common.cuh"
@@ -18,6 +20,16 @@ int sm_count()
         cached[dev] = n;
     }
     return cached[dev];
+}
+
+// MOE_NO_PDL=1 in the environment launches every kernel with plain stream ordering.
+bool pdl_enabled()
+{
+    static const bool on = [] {
+        const char *e = getenv("MOE_NO_PDL");
+        return !(e && e[0] == '1');
+    }();
+    return on;
 }
 
 static thread_local int g_last_launches = 0;
@@ -120,10 +132,7 @@ static thread_local bool g_probe_armed = false;  // only moe_verify_layer arms i
 PlanView plan_view(char *ws, const Workspace &L)
 {
     return PlanView{reinterpret_cast<int32_t *>(ws + L.plan_header),
-                    reinterpret_cast<Segment *>(ws + L.plan_routed),
-                    reinterpret_cast<Segment *>(ws + L.plan_shared),
-                    reinterpret_cast<Segment *>(ws + L.plan_tc_routed),
-                    reinterpret_cast<Segment *>(ws + L.plan_tc_shared)};
+                    reinterpret_cast<Segment *>(ws + L.plan_seg)};
 }
 
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
@@ -137,24 +146,13 @@ moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_b
     __nv_bfloat16 *h = reinterpret_cast<__nv_bfloat16 *>(ws + L.h);
     __nv_bfloat16 *hs = reinterpret_cast<__nv_bfloat16 *>(ws + L.h_shared);
     __nv_bfloat16 *xs = reinterpret_cast<__nv_bfloat16 *>(ws + L.x_sorted);
-    // no group can have more than T rows: below the threshold the tensor-core kernels have
-    // nothing to do and are not launched at all
-    const bool tc = T > TC_MIN_ROWS;
     if (!plan_ready)
-        MOE_STAGE(MOE_STAGE_PLAN,
-                  launch_plan(c, T, offsets, with_shared, TC_MIN_ROWS, status, plan, s));
-    if (tc)
-        MOE_STAGE(MOE_STAGE_GATHER, launch_gather_rows(c, x, perm, T, xs, s));
+        MOE_STAGE(MOE_STAGE_PLAN, launch_plan(c, T, offsets, status, plan, s));
+    MOE_STAGE(MOE_STAGE_GATHER, launch_gather_rows(c, x, perm, T, xs, s));
     MOE_STAGE(MOE_STAGE_GATE_UP,
-              launch_ffn_stream_gateup(c, w, x, T, perm, plan, with_shared, h, hs, s));
-    if (tc)
-        MOE_STAGE(MOE_STAGE_GATE_UP_TC,
-                  launch_ffn_tc_gateup(c, w, x, xs, T, plan, with_shared, h, hs, status, s));
+              launch_ffn_gateup(c, w, x, xs, T, plan, with_shared, h, hs, status, s));
     MOE_STAGE(MOE_STAGE_DOWN,
-              launch_ffn_stream_down(c, w, T, plan, with_shared, h, hs, y, shared_y, s));
-    if (tc)
-        MOE_STAGE(MOE_STAGE_DOWN_TC,
-                  launch_ffn_tc_down(c, w, T, plan, with_shared, h, hs, y, shared_y, status, s));
+              launch_ffn_down(c, w, T, plan, with_shared, h, hs, y, shared_y, status, s));
     return MOE_OK;
 }
 
@@ -330,8 +328,7 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
     const PlanView plan = plan_view(base, L);
     MOE_STAGE(MOE_STAGE_PERMUTE,
               launch_permute(*cfg, topk_idx, T, counts, offsets, perm, inv_perm, active, n_active, s,
-                             &plan, has_shared, TC_MIN_ROWS,
-                             reinterpret_cast<int32_t *>(base + L.status)));
+                             &plan, reinterpret_cast<int32_t *>(base + L.status)));
     st = run_ffn(*cfg, *w, xb, T, offsets, perm, y, ys, base, L, s, launches, true);
     if (st != MOE_OK)
         return st;
@@ -375,7 +372,7 @@ moe_status_t moe_check(void *ws, void *stream)
 
 moe_status_t moe_profile_stage(int32_t stage, void *start_event, void *stop_event)
 {
-    if (stage > MOE_STAGE_DOWN_TC || (stage >= 0 && (!start_event || !stop_event)))
+    if (stage > MOE_STAGE_GATHER || (stage >= 0 && (!start_event || !stop_event)))
         return MOE_ERR_INVALID_ARG;
     g_probe.stage = stage < 0 ? -1 : stage;
     g_probe.start = static_cast<cudaEvent_t>(start_event);

@@ -9,49 +9,30 @@
 namespace moe {
 
 // ---------------------------------------------------------------------------------------
-// Segment plan.  A segment is a run of at most SEG_TOKENS consecutive sorted rows that
-// belong to one group (a routed expert, or the shared expert on rows of x itself).  The
-// plan kernel derives the list from the grouping offsets on the device, so the host never
-// needs the data-dependent counts and no launch waits for a copy.
+// Segment plan.  The token rows of an activated expert (a "group") are cut into segments of
+// at most SEG_TOKENS consecutive sorted rows, the M extent of one tensor-core instruction.
+// The plan lists one entry per segment; every entry carries its whole group, so that any
+// segment index leads to the group, its first segment and its number of segments.  The plan
+// is derived from the grouping offsets on the device: the host never needs the
+// data-dependent counts and no launch waits for a copy.
 // ---------------------------------------------------------------------------------------
-constexpr int SEG_TOKENS = 32;      // rows per segment of the streaming path (4 MMA n-chunks)
-constexpr int TC_SEG_TOKENS = 128;  // rows per segment of the tensor-core path (UMMA N)
-constexpr int TC_MIN_ROWS = 32;     // groups with more rows than this take the tensor-core path
+constexpr int SEG_TOKENS = 128;
 constexpr int PLAN_HEADER_INTS = 16;
 
 struct Segment {
-    int32_t expert;  // routed expert id, or -1 for the shared expert
-    int32_t row0;    // first sorted row (routed) or first token row (shared)
-    int32_t n;       // rows in this segment, 1..SEG_TOKENS
-    int32_t pad;
+    int32_t expert;     // routed expert id of the group
+    int32_t row0;       // first sorted row of the group
+    int32_t n;          // rows of the group (all its segments together)
+    int32_t first_seg;  // plan index of the group's first segment
 };
 
-// plan header (ints): [0] routed / [1] shared streaming segments,
-//                     [2] routed / [3] shared tensor-core segments
+// plan header (ints): [0] number of segments over all activated experts
 struct PlanView {
     int32_t *header;
-    Segment *routed;     // capacity max_routed_segments()
-    Segment *shared;     // capacity max_shared_segments()
-    Segment *tc_routed;  // capacity max_tc_routed_segments()
-    Segment *tc_shared;  // capacity max_tc_shared_segments()
+    Segment *seg;  // capacity max_segments()
 };
 
-__host__ __device__ inline int max_routed_segments(int E, int A)
-{
-    return E + A / SEG_TOKENS + 1;
-}
-__host__ __device__ inline int max_shared_segments(int T)
-{
-    return (T + SEG_TOKENS - 1) / SEG_TOKENS;
-}
-__host__ __device__ inline int max_tc_routed_segments(int E, int A)
-{
-    return E + A / TC_SEG_TOKENS + 1;
-}
-__host__ __device__ inline int max_tc_shared_segments(int T)
-{
-    return (T + TC_SEG_TOKENS - 1) / TC_SEG_TOKENS;
-}
+__host__ __device__ inline int max_segments(int E, int A) { return E + A / SEG_TOKENS + 1; }
 
 // ---------------------------------------------------------------------------------------
 // Workspace layout (every region 256-byte aligned).
@@ -69,11 +50,8 @@ struct Workspace {
     size_t perm;          // i32 [A]
     size_t inv_perm;      // i32 [A]
     size_t plan_header;   // i32 [PLAN_HEADER_INTS]
-    size_t plan_routed;   // Segment[max_routed_segments]
-    size_t plan_shared;   // Segment[max_shared_segments]
-    size_t plan_tc_routed;  // Segment[max_tc_routed_segments]
-    size_t plan_tc_shared;  // Segment[max_tc_shared_segments]
-    size_t x_sorted;      // bf16 [A, H]      token rows in sorted order (tensor-core path)
+    size_t plan_seg;      // Segment[max_segments]
+    size_t x_sorted;      // bf16 [A, H]      token rows in sorted order
     size_t h;             // bf16 [A, I]      SwiGLU intermediate, sorted order
     size_t h_shared;      // bf16 [T, I_s]
     size_t y;             // bf16 [A, H]      expert outputs, sorted order
@@ -105,11 +83,8 @@ inline Workspace workspace_layout(const moe_config_t &c, int T)
     w.perm = take(A * 4);
     w.inv_perm = take(A * 4);
     w.plan_header = take(PLAN_HEADER_INTS * 4);
-    w.plan_routed = take(sizeof(Segment) * (size_t)max_routed_segments((int)E, (int)A));
-    w.plan_shared = take(sizeof(Segment) * (size_t)max_shared_segments(T));
-    w.plan_tc_routed = take(sizeof(Segment) * (size_t)max_tc_routed_segments((int)E, (int)A));
-    w.plan_tc_shared = take(sizeof(Segment) * (size_t)max_tc_shared_segments(T));
-    w.x_sorted = take(T > TC_MIN_ROWS ? A * H * 2 : 0);
+    w.plan_seg = take(sizeof(Segment) * (size_t)max_segments((int)E, (int)A));
+    w.x_sorted = take(A * H * 2);
     w.h = take(A * (size_t)c.inter * 2);
     w.h_shared = take((size_t)T * c.shared_inter * 2);
     w.y = take(A * H * 2);
@@ -133,36 +108,29 @@ cudaError_t launch_route_topk(const moe_config_t &c, const float *logits, int T,
 cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int32_t *counts,
                            int32_t *offsets, int32_t *perm, int32_t *inv_perm, int32_t *active,
                            int32_t *n_active, cudaStream_t s, const PlanView *plan = nullptr,
-                           bool with_shared = false, int tc_min_rows = TC_MIN_ROWS,
                            int32_t *status = nullptr);
-cudaError_t launch_plan(const moe_config_t &c, int T, const int32_t *offsets, bool with_shared,
-                        int tc_min_rows, int32_t *status, PlanView plan, cudaStream_t s);
-// tensor-core path (groups with more than TC_MIN_ROWS rows)
+cudaError_t launch_plan(const moe_config_t &c, int T, const int32_t *offsets, int32_t *status,
+                        PlanView plan, cudaStream_t s);
+// expert FFN on the tensor cores, weights streamed by TMA (every group size):
+// gate/up + SwiGLU -> h[row,:] (routed, sorted order) and h_shared[t,:];
+// down projection  -> y[row,:] and y_shared[t,:]
+cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x,
+                              const __nv_bfloat16 *x_sorted, int T, PlanView plan, bool with_shared,
+                              __nv_bfloat16 *h, __nv_bfloat16 *h_shared, int32_t *status,
+                              cudaStream_t s);
+cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T, PlanView plan,
+                            bool with_shared, const __nv_bfloat16 *h, const __nv_bfloat16 *h_shared,
+                            __nv_bfloat16 *y, __nv_bfloat16 *y_shared, int32_t *status,
+                            cudaStream_t s);
+// token rows in sorted order (the token operand of the routed gate/up tiles)
 cudaError_t launch_gather_rows(const moe_config_t &c, const __nv_bfloat16 *x, const int32_t *perm,
                                int T, __nv_bfloat16 *x_sorted, cudaStream_t s);
-cudaError_t launch_ffn_tc_gateup(const moe_config_t &c, const moe_weights_t &w,
-                                 const __nv_bfloat16 *x, const __nv_bfloat16 *x_sorted, int T,
-                                 PlanView plan, bool with_shared, __nv_bfloat16 *h,
-                                 __nv_bfloat16 *h_shared, int32_t *status, cudaStream_t s);
-cudaError_t launch_ffn_tc_down(const moe_config_t &c, const moe_weights_t &w, int T, PlanView plan,
-                               bool with_shared, const __nv_bfloat16 *h,
-                               const __nv_bfloat16 *h_shared, __nv_bfloat16 *y,
-                               __nv_bfloat16 *y_shared, int32_t *status, cudaStream_t s);
-// gate/up + SwiGLU for every segment of the plan: h[row,:] (routed) and h_shared[row,:]
-cudaError_t launch_ffn_stream_gateup(const moe_config_t &c, const moe_weights_t &w,
-                                     const __nv_bfloat16 *x, int T, const int32_t *perm,
-                                     PlanView plan, bool with_shared, __nv_bfloat16 *h,
-                                     __nv_bfloat16 *h_shared, cudaStream_t s);
-// down projection for every segment: y[row,:] and y_shared[row,:]
-cudaError_t launch_ffn_stream_down(const moe_config_t &c, const moe_weights_t &w, int T,
-                                   PlanView plan, bool with_shared, const __nv_bfloat16 *h,
-                                   const __nv_bfloat16 *h_shared, __nv_bfloat16 *y,
-                                   __nv_bfloat16 *y_shared, cudaStream_t s);
 cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, const int32_t *inv_perm,
                            const float *topk_w, const __nv_bfloat16 *shared_y,
                            const float *shared_scale, int T, __nv_bfloat16 *out, cudaStream_t s);
 
 int sm_count();
+bool pdl_enabled();  // programmatic dependent launch between the layer's kernels
 
 // Host-side argument checks and the FFN launch sequence shared by the entry points.
 bool aligned16(const void *p);
@@ -181,6 +149,26 @@ moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_b
 // Device helpers.
 // ---------------------------------------------------------------------------------------
 #ifdef __CUDACC__
+
+// Launch with the programmatic-stream-serialization attribute: the kernel may begin while its
+// predecessor in the stream is still running and must execute griddepcontrol.wait before it
+// touches anything the predecessor produces.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                              cudaStream_t s, Args &&...args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // 128-bit streaming load: weights are read exactly once, keep them out of L1.
 __device__ __forceinline__ uint4 ld_stream_v4(const void *p)

@@ -1,0 +1,891 @@
+// Expert FFN (gate/up + SwiGLU, and down projection) for every group size: the activated
+// experts' weights are streamed from HBM exactly once by TMA through a ring of shared-memory
+// slots and contracted on the tensor cores (tcgen05.mma, fp32 accumulators in TMEM).
+//
+// Orientation.  A tcgen05.mma of shape M x N x 16 occupies the tensor pipe for about M cycles
+// whatever N is (measured: 146 cycles for M = 128 and any N from 16 to 256).  The weight tile
+// is therefore the N operand (up to 256 rows per instruction: a gate tile and the matching up
+// tile stacked, or 256 rows of W_down) and the group's token rows are the M operand (128 TMEM
+// lanes, of which only the first n carry tokens; the remaining lanes compute on stale shared
+// memory and are never read).  One instruction then retires 8 KB of weights, far more than
+// HBM delivers per SM in that time, so the kernel stays bandwidth-bound from one token per
+// expert up to the roofline ridge (Sec. 3.3: the layer's time is the time to load the
+// activated experts), and at 128 tokens per segment the same instruction runs at full rate.
+//
+// Work partition.  Output features are independent, so the weight rows of all groups are
+// laid end to end and every CTA of the persistent grid takes an equal contiguous share (in
+// units of 16 rows): no tile-count quantisation, no tail wave.  The shared expert's rows and
+// the routed experts' rows are divided separately, so that the shared part -- which depends
+// on nothing the layer computes -- can run before the routing result exists.  Inside its
+// share a CTA cuts tiles of at most 128 (gate/up) or 256 (down) rows; for a group with more
+// than 128 token rows it runs the tile once per 128-row segment, back to back, so that the
+// tile's second and later passes come from L2.
+//
+// A weight slot of the shared-memory ring holds `kboxes` 64-element k boxes of one tile
+// (64 KB for a full tile), so that one producer/consumer hand-shake moves enough bytes to
+// keep HBM busy; the token operand lives in a second ring whose entries are sized by the
+// segment's row count.
+//
+// CTA = 7 warps.  warp 0: weight producer (one lane issues TMA), warp 1: MMA issuer (one
+// lane) and owner of the TMEM allocation, warp 2: token-operand producer, warps 3..6:
+// epilogue (tcgen05.ld of one TMEM lane quarter each, SwiGLU, bf16 store).  Rings and the
+// two accumulator buffers are handed over through mbarriers.  Every wait is bounded: when one
+// gives up it raises the CTA's abort flag and the device status word, all roles leave their
+// loops, TMEM is freed and the kernel returns.
+//
+// Programmatic dependent launch: the kernels may start while their predecessor in the stream
+// is still running.  Work that depends only on the caller's inputs (shared-expert tiles in the
+// gate/up pass, weight prefetch in the down pass) is done before griddepcontrol.wait, so it
+// overlaps the routing kernels; everything produced inside the layer is touched after it.
+#include <cuda.h>
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace moe {
+
+constexpr int FF_THREADS = 224;
+constexpr int FF_MAX_W_SLOTS = 8;
+constexpr int FF_X_ENTRIES = 8;                               // token-ring entries in flight
+constexpr int FF_SEG = SEG_TOKENS;                            // token rows per segment (MMA M)
+constexpr uint64_t FF_WAIT_NS = 1000ull * 1000ull * 1000ull;  // 1 s per wait
+constexpr int FF_TMEM_COLS = 512;
+constexpr int FF_SMEM_LIMIT = 227 * 1024;
+constexpr int FF_X_UNIT = 2048;  // token ring unit: 16 rows x 128 bytes
+constexpr int FF_HEIGHTS = 4;    // TMA box heights for weight tiles: 128, 64, 32, 16 rows
+
+struct FfnArgs {
+    int rows[2];   // output features per group kind (0 routed, 1 shared), multiples of 16
+    int K[2];      // reduction length per group kind
+    __nv_bfloat16 *out[2];
+    int out_ld[2];
+    const int32_t *plan_header;  // [0] = number of segments
+    const Segment *seg;
+    int32_t *status;
+    int T;             // token rows (the shared expert's group)
+    int with_shared;   // shared expert present in this launch
+    int max_tile;      // weight rows per tile: 128 (gate + up stacked) or 256 (down)
+    int kboxes;        // 64-element k boxes per weight slot
+    int w_slot_bytes;  // capacity of a weight slot
+    int n_w_slots;
+    int x_units;       // token ring size in FF_X_UNIT units
+};
+
+// Tensor maps of one pass: weights [kind][matrix][box height], token operand [kind].
+struct FfnMaps {
+    CUtensorMap w[2][2][FF_HEIGHTS];
+    CUtensorMap x[2];
+};
+
+// ---- PTX wrappers ----------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ uint64_t global_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false (and raises the abort flag) if the phase did not complete in
+// FF_WAIT_NS or another role already aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          int32_t *status)
+{
+    if (mbar_try_wait(bar, parity))
+        return true;
+    const uint64_t t0 = global_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity))
+                return true;
+        if (*abort_flag)
+            return false;
+        if (global_ns() - t0 > FF_WAIT_NS) {
+            *abort_flag = 1;
+            atomicExch(status, 1);
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                            int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4}], [%2];"
+        :
+        : "r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+__device__ __forceinline__ void prefetch_map(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Blocks until the preceding kernel in the stream has completed and its writes are visible
+// (returns at once when the kernel was not launched as a programmatic dependent).
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel in the stream start its own prologue.
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        :
+        : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Arrives on the mbarrier when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+          "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr));
+}
+
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7])
+        : "r"(taddr));
+}
+
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) with
+// the 128-byte swizzle TMA wrote: 8-row groups 1024 bytes apart (stride byte offset), leading
+// byte offset unused for swizzled K-major (1), descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr)
+{
+    return (uint64_t)((smem_addr >> 4) & 0x3fffu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+
+// kind::f16 instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n
+// (a multiple of 16, at most 256).
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+// ---- kernel ----------------------------------------------------------------------------
+
+// One work item: one segment of token rows of a group against one tile of its weight rows.
+struct Item {
+    int grp;     // 0 routed, 1 shared
+    int expert;  // routed expert id (0 for the shared expert)
+    int f0;      // first output feature (weight row inside the expert), multiple of 16
+    int h;       // weight rows of the tile, multiple of 16
+    int row0;    // first token row (sorted row for routed groups, token for the shared expert)
+    int n;       // token rows, 1..FF_SEG
+};
+
+// Walks the items of one CTA: its share of the shared expert's rows first (they depend on
+// nothing the layer computes), then its share of the routed groups' rows.  The routed part
+// needs the segment plan, which the preceding kernels write: next() calls
+// griddepcontrol.wait once before it touches the plan (or before reporting the end).
+struct ItemWalk {
+    const FfnArgs &a;
+    const int max_units;
+    // shared expert: row units [su, su_end)
+    int su, su_end, nseg_s;
+    // routed groups: from (fs, u) to (fs_hi, u_hi); fs = plan index of a group's first segment
+    int R0, nseg_total, fs, u, fs_hi, u_hi;
+    bool synced, group_loaded;
+    // current group and tile
+    Segment sg;
+    int g_nseg, g_u_end;
+    bool have_tile;
+    int t_grp, t_expert, t_u0, t_h, t_row0, t_n, t_nseg, t_s;
+
+    __device__ ItemWalk(const FfnArgs &args, bool already_synced)
+        : a(args), max_units(args.max_tile >> 4), synced(false), group_loaded(false), have_tile(false)
+    {
+        const int G = gridDim.x, c = blockIdx.x;
+        const int Us = a.with_shared ? a.rows[1] >> 4 : 0;
+        su = (int)((long long)c * Us / G);
+        su_end = (int)((long long)(c + 1) * Us / G);
+        nseg_s = (a.T + FF_SEG - 1) / FF_SEG;
+        R0 = a.rows[0] >> 4;
+        nseg_total = fs = u = fs_hi = u_hi = 0;
+        if (already_synced)
+            sync(false);
+    }
+    // position p (in units of 16 rows x one segment, groups laid end to end, each group's
+    // units repeated for all its segments) -> (group, row unit)
+    __device__ void boundary(long long p, int &fs_out, int &u_out) const
+    {
+        if (p >= (long long)nseg_total * R0) {
+            fs_out = nseg_total;
+            u_out = 0;
+            return;
+        }
+        const Segment s = a.seg[(int)(p / R0)];
+        const int ns = (s.n + FF_SEG - 1) / FF_SEG;
+        fs_out = s.first_seg;
+        u_out = (int)((p - (long long)s.first_seg * R0) / ns);
+    }
+    __device__ void sync(bool wait)
+    {
+        if (wait)
+            griddep_wait();
+        nseg_total = a.plan_header[0];
+        const long long P = (long long)nseg_total * R0;
+        const int G = gridDim.x, c = blockIdx.x;
+        boundary(P * c / G, fs, u);
+        boundary(P * (c + 1) / G, fs_hi, u_hi);
+        synced = true;
+    }
+    // false when this CTA has no further item
+    __device__ bool next(Item &it)
+    {
+        for (;;) {
+            if (have_tile) {
+                if (t_s < t_nseg) {
+                    it.grp = t_grp;
+                    it.expert = t_expert;
+                    it.f0 = t_u0 << 4;
+                    it.h = t_h << 4;
+                    it.row0 = t_row0 + t_s * FF_SEG;
+                    it.n = min(FF_SEG, t_n - t_s * FF_SEG);
+                    ++t_s;
+                    return true;
+                }
+                have_tile = false;
+            }
+            if (su < su_end) {  // next tile of the shared expert
+                t_h = min(max_units, su_end - su);
+                t_grp = 1;
+                t_expert = 0;
+                t_u0 = su;
+                t_row0 = 0;
+                t_n = a.T;
+                t_nseg = nseg_s;
+                t_s = 0;
+                su += t_h;
+                have_tile = true;
+                continue;
+            }
+            if (!synced)
+                sync(true);
+            if (fs >= nseg_total || (fs == fs_hi && u >= u_hi))
+                return false;
+            if (!group_loaded) {
+                sg = a.seg[fs];
+                g_nseg = (sg.n + FF_SEG - 1) / FF_SEG;
+                g_u_end = fs == fs_hi ? u_hi : R0;
+                group_loaded = true;
+            }
+            if (u < g_u_end) {  // next tile of this group
+                t_h = min(max_units, g_u_end - u);
+                t_grp = 0;
+                t_expert = sg.expert;
+                t_u0 = u;
+                t_row0 = sg.row0;
+                t_n = sg.n;
+                t_nseg = g_nseg;
+                t_s = 0;
+                u += t_h;
+                have_tile = true;
+                continue;
+            }
+            fs += g_nseg;  // group done: on to the next one
+            u = 0;
+            group_loaded = false;
+        }
+    }
+};
+
+// Placement of the token-ring entries.  An entry takes `m` consecutive units and never wraps:
+// when it does not fit before the end of the ring it starts at unit 0.  Producer and MMA
+// issuer replay the same sequence of sizes, so they agree on every position.
+struct XRingWalk {
+    int units, cur, count;
+    __device__ XRingWalk(int n_units) : units(n_units), cur(0), count(0) {}
+    // returns the first unit of the next entry; `pad` = units skipped at the end of the ring
+    __device__ int place(int m, int &pad)
+    {
+        pad = 0;
+        if (cur + m > units) {
+            pad = units - cur;  // may be 0 when the previous entry ended exactly at the end
+            cur = 0;
+        }
+        const int at = cur;
+        cur += m;
+        ++count;
+        return at;
+    }
+};
+
+__device__ __forceinline__ int pieces16(int n) { return (n + 15) >> 4; }
+
+template <bool GATED>
+__device__ __forceinline__ void epilogue_store8(const uint32_t *g, const uint32_t *u,
+                                                __nv_bfloat16 *dst)
+{
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float a = __uint_as_float(g[2 * j]), b = __uint_as_float(g[2 * j + 1]);
+        if (GATED) {
+            a = silu_f(a) * __uint_as_float(u[2 * j]);
+            b = silu_f(b) * __uint_as_float(u[2 * j + 1]);
+        }
+        __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+        o[j] = *reinterpret_cast<uint32_t *>(&p);
+    }
+    *reinterpret_cast<uint4 *>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// GATED: W_gate and W_up tiles -> h = silu(g) * u.   !GATED: W_down tiles -> y.
+template <bool GATED>
+__global__ void __launch_bounds__(FF_THREADS, 1)
+ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
+{
+    constexpr int ACC_COLS = 256;      // TMEM columns per accumulator buffer
+    constexpr int NW = GATED ? 2 : 1;  // weight matrices stacked in one N operand
+
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[2 * FF_MAX_W_SLOTS + 2 * FF_X_ENTRIES + 4];
+    __shared__ uint32_t tmem_base_holder;
+    __shared__ int abort_flag;
+
+    const int NS = args.n_w_slots;
+    const int kb = args.kboxes;
+    // token ring first: an MMA reads 128 token rows from an entry that may hold fewer, and
+    // the excess of the last entry then falls into the weight ring instead of past the end
+    const uint32_t ring_x = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle needs 1 KB alignment
+    const uint32_t ring_w = ring_x + (uint32_t)args.x_units * FF_X_UNIT;
+    const uint32_t bar0 = smem_u32(bars);
+    auto w_full = [&](int s) { return bar0 + 8u * s; };
+    auto w_empty = [&](int s) { return bar0 + 8u * (FF_MAX_W_SLOTS + s); };
+    auto x_full = [&](int s) { return bar0 + 8u * (2 * FF_MAX_W_SLOTS + s); };
+    auto x_empty = [&](int s) { return bar0 + 8u * (2 * FF_MAX_W_SLOTS + FF_X_ENTRIES + s); };
+    auto acc_full = [&](int b) { return bar0 + 8u * (2 * FF_MAX_W_SLOTS + 2 * FF_X_ENTRIES + b); };
+    auto acc_empty = [&](int b) { return bar0 + 8u * (2 * FF_MAX_W_SLOTS + 2 * FF_X_ENTRIES + 2 + b); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(w_full(s), 1);
+            mbar_init(w_empty(s), 1);
+        }
+        for (int s = 0; s < FF_X_ENTRIES; ++s) {
+            mbar_init(x_full(s), 1);
+            mbar_init(x_empty(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(acc_full(b), 1);
+            mbar_init(acc_empty(b), 4);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(&tmem_base_holder)),
+                     "r"(FF_TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_holder;
+    volatile int *abortp = &abort_flag;
+
+    if (warp == 0) {
+        // ---------------- weight producer ----------------
+        if (lane == 0) {
+            // gate/up pass: the shared expert's weights and x are the caller's inputs, so those
+            // items run before the wait.  Down pass: every weight tile may be fetched ahead --
+            // the launch order guarantees that the plan is complete when this kernel starts.
+            ItemWalk walk(args, !GATED);
+            bool launched = !GATED;
+            if (!GATED)
+                griddep_launch();
+            int slot = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            Item it;
+            while (ok && walk.next(it)) {
+                if (!launched && walk.synced) {
+                    griddep_launch();  // after the wait: dependents may rely on the plan
+                    launched = true;
+                }
+                const int K = args.K[it.grp];
+                const uint32_t tile_bytes = (uint32_t)it.h * 128u;
+                const int wrow = it.expert * args.rows[0] + it.f0;  // expert = 0 for the shared kind
+                for (int k0 = 0; k0 < K; k0 += 64 * kb) {
+                    const int nbox = min(kb, (K - k0 + 63) >> 6);
+                    if (!mbar_wait(w_empty(slot), phase ^ 1u, abortp, args.status)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t base = ring_w + slot * args.w_slot_bytes;
+                    mbar_expect_tx(w_full(slot), nbox * NW * tile_bytes);
+                    for (int b = 0; b < nbox; ++b) {
+#pragma unroll
+                        for (int m = 0; m < NW; ++m) {
+                            // the tile as boxes of 128, 64, 32 and 16 rows, stacked
+                            uint32_t dst = base + (uint32_t)(b * NW + m) * tile_bytes;
+                            int row = wrow, rem = it.h;
+                            while (rem > 0) {
+                                const int hi = rem >= 128 ? 0 : (rem >= 64 ? 1 : (rem >= 32 ? 2 : 3));
+                                const int bh = 128 >> hi;
+                                tma_load_2d(dst, &maps.w[it.grp][m][hi], w_full(slot), k0 + 64 * b, row);
+                                dst += (uint32_t)bh * 128u;
+                                row += bh;
+                                rem -= bh;
+                            }
+                        }
+                    }
+                    if (++slot == NS) {
+                        slot = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+            if (!walk.synced)
+                walk.sync(true);
+            if (!launched)
+                griddep_launch();
+            if (!ok) {
+                // copies already issued may still be landing: give them time before teardown
+                const uint64_t t0 = global_ns();
+                while (global_ns() - t0 < 1000000ull) {
+                }
+            }
+        }
+    } else if (warp == 2) {
+        // ---------------- token-operand producer ----------------
+        if (lane == 0) {
+            // down pass: h is written by the preceding kernel
+            if (!GATED)
+                griddep_wait();
+            ItemWalk walk(args, !GATED);
+            XRingWalk ring(args.x_units);
+            int released = 0;          // entries known to have been consumed
+            int v_cur = 0, v_rel = 0;  // virtual unit positions: issued up to / released up to
+            int v_end_of[FF_X_ENTRIES];
+            bool ok = true;
+            Item it;
+            while (ok && walk.next(it)) {
+                const CUtensorMap *mx = &maps.x[it.grp];
+                const int K = args.K[it.grp];
+                const int pieces = pieces16(it.n);
+                const int m = pieces * kb;
+                for (int k0 = 0; k0 < K; k0 += 64 * kb) {
+                    const int nbox = min(kb, (K - k0 + 63) >> 6);
+                    const int j = ring.count;
+                    int pad;
+                    const int at = ring.place(m, pad);
+                    const int v_end = v_cur + pad + m;
+                    // the entry's units (and its barrier pair) must have been released
+                    // (with nothing outstanding the whole ring is free, padding included)
+                    while (released < j &&
+                           (j - released >= FF_X_ENTRIES || v_end - v_rel > args.x_units)) {
+                        const int r = released % FF_X_ENTRIES;
+                        if (!mbar_wait(x_empty(r), (uint32_t)(released / FF_X_ENTRIES) & 1u, abortp,
+                                       args.status)) {
+                            ok = false;
+                            break;
+                        }
+                        v_rel = v_end_of[r];
+                        ++released;
+                    }
+                    if (!ok)
+                        break;
+                    const int e = j % FF_X_ENTRIES;
+                    v_end_of[e] = v_end;
+                    v_cur = v_end;
+                    const uint32_t base = ring_x + (uint32_t)at * FF_X_UNIT;
+                    mbar_expect_tx(x_full(e), (uint32_t)(nbox * pieces) * FF_X_UNIT);
+                    for (int b = 0; b < nbox; ++b)
+                        for (int p = 0; p < pieces; ++p)
+                            tma_load_2d(base + (uint32_t)(b * pieces + p) * FF_X_UNIT, mx, x_full(e),
+                                        k0 + 64 * b, it.row0 + 16 * p);
+                }
+            }
+            if (!walk.synced)
+                walk.sync(true);
+            if (!ok) {
+                const uint64_t t0 = global_ns();
+                while (global_ns() - t0 < 1000000ull) {
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            ItemWalk walk(args, !GATED);
+            XRingWalk ring(args.x_units);
+            int sw = 0;
+            uint32_t pw = 0;
+            bool ok = true;
+            int n_items = 0;
+            Item it;
+            while (ok && walk.next(it)) {
+                const int buf = n_items & 1;
+                const uint32_t acc_phase = (uint32_t)(n_items >> 1) & 1u;
+                ++n_items;
+                if (!mbar_wait(acc_empty(buf), acc_phase ^ 1u, abortp, args.status))
+                    break;
+                tc_fence_after();
+                const uint32_t tile_bytes = (uint32_t)it.h * 128u;
+                const uint32_t idesc = umma_idesc_bf16(NW * it.h);
+                const uint32_t d0 = tmem_base + (uint32_t)(buf * ACC_COLS);
+                const int K = args.K[it.grp];
+                const int pieces = pieces16(it.n);
+                const int m = pieces * kb;
+                for (int k0 = 0; k0 < K; k0 += 64 * kb) {
+                    const int nbox = min(kb, (K - k0 + 63) >> 6);
+                    const int j = ring.count;
+                    int pad;
+                    const int at = ring.place(m, pad);
+                    const int e = j % FF_X_ENTRIES;
+                    if (!mbar_wait(x_full(e), (uint32_t)(j / FF_X_ENTRIES) & 1u, abortp, args.status) ||
+                        !mbar_wait(w_full(sw), pw, abortp, args.status)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t xbase = ring_x + (uint32_t)at * FF_X_UNIT;
+                    const uint32_t wbase = ring_w + sw * args.w_slot_bytes;
+                    for (int b = 0; b < nbox; ++b) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const uint32_t accum = (k0 | b | q) != 0 ? 1u : 0u;
+                            umma_bf16(d0, umma_desc_sw128(xbase + (uint32_t)(b * pieces) * FF_X_UNIT + q * 32),
+                                      umma_desc_sw128(wbase + b * NW * tile_bytes + q * 32), idesc, accum);
+                        }
+                    }
+                    umma_commit(w_empty(sw));  // reusable once these MMAs have read them
+                    umma_commit(x_empty(e));
+                    if (++sw == NS) {
+                        sw = 0;
+                        pw ^= 1u;
+                    }
+                }
+                if (ok)
+                    umma_commit(acc_full(buf));  // accumulator complete
+            }
+            if (!walk.synced)
+                walk.sync(true);
+        }
+    } else {
+        // ---------------- epilogue (warps 3..6) ----------------
+        // down pass: everything this kernel writes or reads besides weights belongs to the
+        // layer call in flight, so it waits for the preceding kernel first
+        if (!GATED)
+            griddep_wait();
+        const int quarter = warp & 3;  // TMEM lanes 32*quarter .. +31 belong to this warp
+        ItemWalk walk(args, !GATED);
+        int n_items = 0;
+        Item it;
+        for (;;) {
+            // the walk is identical in all lanes; griddepcontrol.wait inside next() is
+            // executed by every lane
+            if (!walk.next(it))
+                break;
+            const int buf = n_items & 1;
+            const uint32_t acc_phase = (uint32_t)(n_items >> 1) & 1u;
+            ++n_items;
+            // every lane waits; the vote makes the decision uniform and reconverges the warp
+            // for the warp-collective tcgen05.ld below
+            const bool ready = mbar_wait(acc_full(buf), acc_phase, abortp, args.status);
+            if (!__all_sync(0xffffffffu, ready))
+                break;
+            tc_fence_after();
+            if (quarter * 32 < it.n) {
+                const int trow = quarter * 32 + lane;  // token row of this thread
+                const bool row_ok = trow < it.n;
+                __nv_bfloat16 *out = args.out[it.grp] + (size_t)(it.row0 + trow) * args.out_ld[it.grp] + it.f0;
+                const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * ACC_COLS);
+                for (int c = 0; c < it.h; c += 16) {
+                    uint32_t g[16], u[16];
+                    tmem_ld16(t0 + c, g);
+                    if (GATED)
+                        tmem_ld16(t0 + it.h + c, u);
+                    tmem_ld_wait();
+                    if (row_ok) {
+                        epilogue_store8<GATED>(g, u, out + c);
+                        epilogue_store8<GATED>(g + 8, u + 8, out + c + 8);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0)
+                mbar_arrive(acc_empty(buf));
+        }
+        if (!walk.synced)
+            walk.sync(true);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();  // lane 0 arrived from the issue loop: reconverge for the aligned dealloc
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                     "r"(FF_TMEM_COLS)
+                     : "memory");
+    }
+}
+
+// ---- gather of the token rows into sorted order (B operand of the gate/up pass) ---------
+
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__restrict__ perm, int A,
+                   int H, int top_k, __nv_bfloat16 *__restrict__ x_sorted)
+{
+    griddep_launch();
+    griddep_wait();
+    const int vec_per_row = H >> 3;
+    const size_t total = (size_t)A * vec_per_row;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total;
+         i += (size_t)gridDim.x * blockDim.x) {
+        const int r = (int)(i / vec_per_row);
+        const int v = (int)(i - (size_t)r * vec_per_row);
+        const int t = perm[r] / top_k;
+        reinterpret_cast<uint4 *>(x_sorted + (size_t)r * H)[v] =
+            reinterpret_cast<const uint4 *>(x + (size_t)t * H)[v];
+    }
+}
+
+cudaError_t launch_gather_rows(const moe_config_t &c, const __nv_bfloat16 *x, const int32_t *perm,
+                               int T, __nv_bfloat16 *x_sorted, cudaStream_t s)
+{
+    const int A = T * c.top_k;
+    const size_t total = (size_t)A * (c.hidden >> 3);
+    size_t blocks = (total + 255) / 256;
+    const size_t cap = (size_t)sm_count() * 8;
+    if (blocks > cap)
+        blocks = cap;
+    return launch_pdl(gather_rows_kernel, dim3((unsigned)blocks), dim3(256), 0, s, x, perm, A,
+                      c.hidden, c.top_k, x_sorted);
+}
+
+// ---- host side: geometry, tensor maps and launches ---------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// 2-D bf16 tensor [rows, cols] (cols contiguous), box = 64 columns x box_rows, 128-byte swizzle.
+static bool make_map(CUtensorMap *m, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn)
+        return false;
+    if (base == nullptr || rows == 0 || cols == 0) {
+        memset(m, 0, sizeof *m);  // group kind not present: never used by the kernel
+        return true;
+    }
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// the four box heights of one weight matrix
+static bool make_weight_maps(CUtensorMap (&m)[FF_HEIGHTS], const void *base, uint64_t rows, uint64_t cols)
+{
+    for (int i = 0; i < FF_HEIGHTS; ++i)
+        if (!make_map(&m[i], base, rows, cols, 128u >> i))
+            return false;
+    return true;
+}
+
+// Expected number of activated experts for T tokens (Eq. N(t): E(1 - (1 - K/E)^T)); the host
+// never sees the routing result, so it sizes the rings from the expected rows per expert.
+static double expected_active_experts(int E, int k, int T)
+{
+    return E * (1.0 - pow(1.0 - (double)k / E, (double)T));
+}
+
+// Ring geometry.  While the expected rows per expert are few the pass is a weight stream:
+// 64 KB weight slots (two k boxes of a full tile) and a small token ring.  Near and beyond
+// the ridge the token operand is as large as the weight tile: one k box per slot and a token
+// ring that holds several 128-row entries.
+static void ffn_geometry(const moe_config_t &c, int T, FfnArgs &a)
+{
+    const double per_group = (double)T * c.top_k / expected_active_experts(c.n_experts, c.top_k, T);
+    const bool streaming = per_group <= 48.0;
+    a.kboxes = streaming ? 2 : 1;
+    a.w_slot_bytes = 256 * 128 * a.kboxes;  // a full tile: 256 stacked rows per k box
+    const int x_ring_bytes = streaming ? 32 * 1024 : 96 * 1024;
+    a.x_units = x_ring_bytes / FF_X_UNIT;
+    const int avail = FF_SMEM_LIMIT - 1024 - 512;  // alignment slack, static shared memory
+    int ns = (avail - x_ring_bytes) / a.w_slot_bytes;
+    if (ns > FF_MAX_W_SLOTS)
+        ns = FF_MAX_W_SLOTS;
+    a.n_w_slots = ns;
+}
+
+template <bool GATED>
+static cudaError_t launch_ffn(FfnArgs &a, const FfnMaps &maps, cudaStream_t s)
+{
+    static bool configured[2] = {false, false};
+    if (!configured[GATED]) {
+        cudaError_t e = cudaFuncSetAttribute(ffn_fused_kernel<GATED>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             FF_SMEM_LIMIT - 512);
+        if (e != cudaSuccess)
+            return e;
+        configured[GATED] = true;
+    }
+    // the 128-row read of the last token entry may run 16 KB past the token ring: the weight
+    // ring behind it is always larger than that
+    const size_t smem = (size_t)a.x_units * FF_X_UNIT + (size_t)a.n_w_slots * a.w_slot_bytes + 1024;
+    if (a.n_w_slots < 2 || smem > FF_SMEM_LIMIT - 512)
+        return cudaErrorInvalidConfiguration;
+    return launch_pdl(ffn_fused_kernel<GATED>, dim3(sm_count()), dim3(FF_THREADS), smem, s, a, maps);
+}
+
+cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x,
+                              const __nv_bfloat16 *x_sorted, int T, PlanView plan, bool with_shared,
+                              __nv_bfloat16 *h, __nv_bfloat16 *h_shared, int32_t *status,
+                              cudaStream_t s)
+{
+    const uint64_t A = (uint64_t)T * c.top_k, H = c.hidden, E = c.n_experts;
+    FfnArgs a{};
+    a.rows[0] = c.inter;
+    a.rows[1] = c.shared_inter;
+    a.K[0] = a.K[1] = c.hidden;
+    a.max_tile = 128;
+    ffn_geometry(c, T, a);
+    FfnMaps maps;
+    memset(&maps, 0, sizeof maps);
+    bool ok = make_weight_maps(maps.w[0][0], w.w_gate, E * c.inter, H) &&
+              make_weight_maps(maps.w[0][1], w.w_up, E * c.inter, H) &&
+              make_map(&maps.x[0], x_sorted, A, H, 16);
+    if (with_shared)
+        ok = ok && make_weight_maps(maps.w[1][0], w.ws_gate, c.shared_inter, H) &&
+             make_weight_maps(maps.w[1][1], w.ws_up, c.shared_inter, H) &&
+             make_map(&maps.x[1], x, T, H, 16);
+    if (!ok)
+        return cudaErrorInvalidValue;
+    a.out[0] = h;
+    a.out[1] = h_shared;
+    a.out_ld[0] = c.inter;
+    a.out_ld[1] = c.shared_inter;
+    a.plan_header = plan.header;
+    a.seg = plan.seg;
+    a.status = status;
+    a.T = T;
+    a.with_shared = with_shared ? 1 : 0;
+    return launch_ffn<true>(a, maps, s);
+}
+
+cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T, PlanView plan,
+                            bool with_shared, const __nv_bfloat16 *h, const __nv_bfloat16 *h_shared,
+                            __nv_bfloat16 *y, __nv_bfloat16 *y_shared, int32_t *status,
+                            cudaStream_t s)
+{
+    const uint64_t A = (uint64_t)T * c.top_k, H = c.hidden, E = c.n_experts;
+    FfnArgs a{};
+    a.rows[0] = a.rows[1] = c.hidden;
+    a.K[0] = c.inter;
+    a.K[1] = c.shared_inter;
+    a.max_tile = 256;
+    ffn_geometry(c, T, a);
+    FfnMaps maps;
+    memset(&maps, 0, sizeof maps);
+    bool ok = make_weight_maps(maps.w[0][0], w.w_down, E * H, c.inter) &&
+              make_map(&maps.x[0], h, A, c.inter, 16);
+    if (with_shared)
+        ok = ok && make_weight_maps(maps.w[1][0], w.ws_down, H, c.shared_inter) &&
+             make_map(&maps.x[1], h_shared, T, c.shared_inter, 16);
+    if (!ok)
+        return cudaErrorInvalidValue;
+    a.out[0] = y;
+    a.out[1] = y_shared;
+    a.out_ld[0] = a.out_ld[1] = c.hidden;
+    a.plan_header = plan.header;
+    a.seg = plan.seg;
+    a.status = status;
+    a.T = T;
+    a.with_shared = with_shared ? 1 : 0;
+    return launch_ffn<false>(a, maps, s);
+}
+
+}  // namespace moe

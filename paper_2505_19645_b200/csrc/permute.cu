@@ -31,56 +31,33 @@ __device__ void block_exclusive_scan(int *vals, int *tmp, int n, int *total)
     __syncthreads();
 }
 
-// Segment plan from per-expert counts and offsets held in shared memory.  A group (expert, or
-// the shared expert with its T rows) with at most tc_min_rows rows is cut into streaming
-// segments of <= SEG_TOKENS rows; a larger group into tensor-core segments of <= TC_SEG_TOKENS
-// rows.  All threads of the block must call it; scan/tmp/total are shared scratch.
+// Segment plan from per-expert counts and offsets held in shared memory: one entry per
+// segment of SEG_TOKENS rows of every activated expert, in ascending expert order.  All
+// threads of the block must call it; scan/tmp/total are shared scratch.
 __device__ void build_plan(const int *cnt_sh, const int *off_sh, int *scan, int *tmp, int *total,
-                           int E, int T, int with_shared, int tc_min_rows, int32_t *status,
-                           PlanView plan)
+                           int E, int32_t *status, PlanView plan)
 {
     const int tid = threadIdx.x;
     const int cnt = tid < E ? cnt_sh[tid] : 0;
     const int row0 = tid < E ? off_sh[tid] : 0;
-    const bool tc = cnt > tc_min_rows;
-    for (int pass = 0; pass < 2; ++pass) {
-        const int seg_rows = pass == 0 ? SEG_TOKENS : TC_SEG_TOKENS;
-        const bool mine = cnt > 0 && (pass == 0 ? !tc : tc);
-        __syncthreads();
-        if (tid < MOE_MAX_EXPERTS)
-            scan[tid] = mine ? (cnt + seg_rows - 1) / seg_rows : 0;
-        __syncthreads();
-        block_exclusive_scan(scan, tmp, E, total);
-        Segment *list = pass == 0 ? plan.routed : plan.tc_routed;
-        if (mine) {
-            int at = scan[tid];
-            for (int r = 0; r < cnt; r += seg_rows) {
-                Segment sg;
-                sg.expert = tid;
-                sg.row0 = row0 + r;
-                sg.n = min(seg_rows, cnt - r);
-                sg.pad = 0;
-                list[at++] = sg;
-            }
-        }
-        if (tid == 0)
-            plan.header[pass == 0 ? 0 : 2] = *total;
-    }
-    const bool shared_tc = T > tc_min_rows;
-    const int seg_rows = shared_tc ? TC_SEG_TOKENS : SEG_TOKENS;
-    const int n_shared = with_shared ? (T + seg_rows - 1) / seg_rows : 0;
-    Segment *slist = shared_tc ? plan.tc_shared : plan.shared;
-    for (int i = tid; i < n_shared; i += blockDim.x) {
+    const int nseg = (cnt + SEG_TOKENS - 1) / SEG_TOKENS;
+    __syncthreads();
+    if (tid < MOE_MAX_EXPERTS)
+        scan[tid] = nseg;
+    __syncthreads();
+    block_exclusive_scan(scan, tmp, E, total);
+    if (nseg > 0) {
+        const int first = scan[tid];
         Segment sg;
-        sg.expert = -1;
-        sg.row0 = i * seg_rows;
-        sg.n = min(seg_rows, T - i * seg_rows);
-        sg.pad = 0;
-        slist[i] = sg;
+        sg.expert = tid;
+        sg.row0 = row0;
+        sg.n = cnt;
+        sg.first_seg = first;
+        for (int i = 0; i < nseg; ++i)
+            plan.seg[first + i] = sg;
     }
     if (tid == 0) {
-        plan.header[1] = shared_tc ? 0 : n_shared;
-        plan.header[3] = shared_tc ? n_shared : 0;
+        plan.header[0] = *total;
         status[0] = 0;  // device status word: cleared at the start of every FFN pass
     }
 }
@@ -94,8 +71,7 @@ __global__ void __launch_bounds__(PERM_THREADS)
 permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__restrict__ counts,
                int32_t *__restrict__ offsets, int32_t *__restrict__ perm,
                int32_t *__restrict__ inv_perm, int32_t *__restrict__ active,
-               int32_t *__restrict__ n_active, int T, int with_shared, int tc_min_rows,
-               int32_t *__restrict__ status, PlanView plan)
+               int32_t *__restrict__ n_active, int32_t *__restrict__ status, PlanView plan)
 {
     __shared__ int hist[MOE_MAX_EXPERTS];
     __shared__ int offs[MOE_MAX_EXPERTS];
@@ -136,7 +112,7 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
         if (tid == 0)
             n_active[0] = total;
         if (plan.header != nullptr)
-            build_plan(hist, offs, flag, tmp, &total, E, T, with_shared, tc_min_rows, status, plan);
+            build_plan(hist, offs, flag, tmp, &total, E, status, plan);
     }
 
     const int warp = tid >> 5, lane = tid & 31;
@@ -169,8 +145,7 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
 
 cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int32_t *counts,
                            int32_t *offsets, int32_t *perm, int32_t *inv_perm, int32_t *active,
-                           int32_t *n_active, cudaStream_t s, const PlanView *plan,
-                           bool with_shared, int tc_min_rows, int32_t *status)
+                           int32_t *n_active, cudaStream_t s, const PlanView *plan, int32_t *status)
 {
     const int E = c.n_experts;
     const int blocks = (E + 31) / 32;
@@ -178,15 +153,13 @@ cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int
     if (plan)
         pv = *plan;
     permute_kernel<<<blocks, PERM_THREADS, 0, s>>>(idx, T * c.top_k, E, counts, offsets, perm,
-                                                   inv_perm, active, n_active, T,
-                                                   with_shared ? 1 : 0, tc_min_rows, status, pv);
+                                                   inv_perm, active, n_active, status, pv);
     return cudaGetLastError();
 }
 
 // Stand-alone plan (moe_grouped_swiglu gets its offsets from the caller).
 __global__ void __launch_bounds__(MOE_MAX_EXPERTS)
-plan_kernel(const int32_t *__restrict__ offsets, int E, int T, int with_shared, int tc_min_rows,
-            int32_t *__restrict__ status, PlanView plan)
+plan_kernel(const int32_t *__restrict__ offsets, int E, int32_t *__restrict__ status, PlanView plan)
 {
     __shared__ int cnt[MOE_MAX_EXPERTS];
     __shared__ int offs[MOE_MAX_EXPERTS];
@@ -202,14 +175,14 @@ plan_kernel(const int32_t *__restrict__ offsets, int E, int T, int with_shared, 
     cnt[tid] = n;
     offs[tid] = row0;
     __syncthreads();
-    build_plan(cnt, offs, scan, tmp, &total, E, T, with_shared, tc_min_rows, status, plan);
+    build_plan(cnt, offs, scan, tmp, &total, E, status, plan);
 }
 
-cudaError_t launch_plan(const moe_config_t &c, int T, const int32_t *offsets, bool with_shared,
-                        int tc_min_rows, int32_t *status, PlanView plan, cudaStream_t s)
+cudaError_t launch_plan(const moe_config_t &c, int T, const int32_t *offsets, int32_t *status,
+                        PlanView plan, cudaStream_t s)
 {
-    plan_kernel<<<1, MOE_MAX_EXPERTS, 0, s>>>(offsets, c.n_experts, T, with_shared ? 1 : 0,
-                                              tc_min_rows, status, plan);
+    (void)T;
+    plan_kernel<<<1, MOE_MAX_EXPERTS, 0, s>>>(offsets, c.n_experts, status, plan);
     return cudaGetLastError();
 }
 
