@@ -12,19 +12,20 @@
 // expert up to the roofline ridge (Sec. 3.3: the layer's time is the time to load the
 // activated experts), and at 128 tokens per segment the same instruction runs at full rate.
 //
-// Work partition.  Output features are independent, so the weight rows of all groups are
-// laid end to end and every CTA of the persistent grid takes an equal contiguous share (in
-// units of 16 rows): no tile-count quantisation, no tail wave.  The shared expert's rows and
-// the routed experts' rows are divided separately, so that the shared part -- which depends
-// on nothing the layer computes -- can run before the routing result exists.  Inside its
-// share a CTA cuts tiles of at most 128 (gate/up) or 256 (down) rows; for a group with more
-// than 128 token rows it runs the tile once per 128-row segment, back to back, so that the
-// tile's second and later passes come from L2.
+// Work partition.  Output features are independent, so the weight rows of all routed
+// groups are laid end to end (one position = 16 rows of one group for one of its 128-row
+// segments) and every CTA of the persistent grid takes one contiguous range: no tile-count
+// quantisation, no tail wave.  The shared expert's rows are cut into full-height tiles that
+// are dealt round-robin to the CTAs; they depend on nothing the layer computes, so they run
+// before the routing result exists, and the routed ranges are then sized so that
+// shared + routed cost is level across the grid.  Inside its range a CTA cuts tiles of at
+// most 128 (gate/up) or 256 (down) rows; for a group with more than 128 token rows it runs
+// the tile once per segment, back to back, so that the second and later passes come from L2.
 //
 // A weight slot of the shared-memory ring holds `kboxes` 64-element k boxes of one tile
-// (64 KB for a full tile), so that one producer/consumer hand-shake moves enough bytes to
-// keep HBM busy; the token operand lives in a second ring whose entries are sized by the
-// segment's row count.
+// (32 KB per box for a full tile), so that one producer/consumer hand-shake moves enough
+// bytes to keep HBM busy; the token operand lives in a second ring whose entries are sized
+// by the segment's row count.
 //
 // CTA = 7 warps.  warp 0: weight producer (one lane issues TMA), warp 1: MMA issuer (one
 // lane) and owner of the TMEM allocation, warp 2: token-operand producer, warps 3..6:
@@ -65,6 +66,8 @@ struct FfnArgs {
     int32_t *status;
     int T;             // token rows (the shared expert's group)
     int with_shared;   // shared expert present in this launch
+    int shared_tiles;  // tiles of the shared expert's rows, dealt round-robin to the CTAs;
+                       // the first (units % tiles) of them have one 16-row unit more
     int max_tile;      // weight rows per tile: 128 (gate + up stacked) or 256 (down)
     int kboxes;        // 64-element k boxes per weight slot
     int w_slot_bytes;  // capacity of a weight slot
@@ -238,15 +241,15 @@ struct Item {
     int n;       // token rows, 1..FF_SEG
 };
 
-// Walks the items of one CTA: its share of the shared expert's rows first (they depend on
-// nothing the layer computes), then its share of the routed groups' rows.  The routed part
-// needs the segment plan, which the preceding kernels write: next() calls
-// griddepcontrol.wait once before it touches the plan (or before reporting the end).
+// Walks the items of one CTA: its tiles of the shared expert first (they depend on nothing
+// the layer computes), then its range of the routed groups' rows.  The routed part needs the
+// segment plan, which the preceding kernels write: next() calls griddepcontrol.wait once
+// before it touches the plan (or before reporting the end).
 struct ItemWalk {
     const FfnArgs &a;
     const int max_units;
-    // shared expert: row units [su, su_end)
-    int su, su_end, nseg_s;
+    // shared expert: tiles sj, sj + grid, ...
+    int sj, Us, s_base, s_rem, nseg_s;
     // routed groups: from (fs, u) to (fs_hi, u_hi); fs = plan index of a group's first segment
     int R0, nseg_total, fs, u, fs_hi, u_hi;
     bool synced, group_loaded;
@@ -259,15 +262,34 @@ struct ItemWalk {
     __device__ ItemWalk(const FfnArgs &args, bool already_synced)
         : a(args), max_units(args.max_tile >> 4), synced(false), group_loaded(false), have_tile(false)
     {
-        const int G = gridDim.x, c = blockIdx.x;
-        const int Us = a.with_shared ? a.rows[1] >> 4 : 0;
-        su = (int)((long long)c * Us / G);
-        su_end = (int)((long long)(c + 1) * Us / G);
+        Us = a.with_shared ? a.rows[1] >> 4 : 0;
+        s_base = a.shared_tiles ? Us / a.shared_tiles : 0;
+        s_rem = a.shared_tiles ? Us % a.shared_tiles : 0;
+        sj = blockIdx.x;
         nseg_s = (a.T + FF_SEG - 1) / FF_SEG;
         R0 = a.rows[0] >> 4;
         nseg_total = fs = u = fs_hi = u_hi = 0;
         if (already_synced)
             sync(false);
+    }
+    // First routed position of CTA c.  CTAs [0, r) hold one shared tile more than CTAs [r, G);
+    // the routed positions first fill the second class up to the first, the rest is spread
+    // over everybody.  Costs are counted in (16 rows x 1 k element x 1 segment): a routed
+    // position costs K[0], a shared unit K[1] * nseg_s.  Integer arithmetic only, so every
+    // role of every CTA derives the same bounds.
+    __device__ long long routed_bound(int c, long long P) const
+    {
+        const int G = gridDim.x;
+        const int r = a.shared_tiles % G;
+        if (r == 0)
+            return P * c / G;
+        const long long tile_cost = (long long)(s_base + (s_rem ? 1 : 0)) * a.K[1] * nseg_s;
+        const long long p_cost = P * a.K[0];
+        const int n_lo = G - r;
+        if (p_cost <= tile_cost * n_lo)
+            return c < r ? 0 : P * (c - r) / n_lo;
+        const long long extra = p_cost - tile_cost * n_lo;  // spread over all G CTAs
+        return (extra * c + tile_cost * G * (c > r ? c - r : 0)) / ((long long)G * a.K[0]);
     }
     // position p (in units of 16 rows x one segment, groups laid end to end, each group's
     // units repeated for all its segments) -> (group, row unit)
@@ -289,9 +311,8 @@ struct ItemWalk {
             griddep_wait();
         nseg_total = a.plan_header[0];
         const long long P = (long long)nseg_total * R0;
-        const int G = gridDim.x, c = blockIdx.x;
-        boundary(P * c / G, fs, u);
-        boundary(P * (c + 1) / G, fs_hi, u_hi);
+        boundary(routed_bound(blockIdx.x, P), fs, u);
+        boundary(routed_bound(blockIdx.x + 1, P), fs_hi, u_hi);
         synced = true;
     }
     // false when this CTA has no further item
@@ -311,16 +332,16 @@ struct ItemWalk {
                 }
                 have_tile = false;
             }
-            if (su < su_end) {  // next tile of the shared expert
-                t_h = min(max_units, su_end - su);
+            if (sj < a.shared_tiles) {  // next tile of the shared expert
+                t_u0 = sj * s_base + min(sj, s_rem);
+                t_h = s_base + (sj < s_rem ? 1 : 0);
                 t_grp = 1;
                 t_expert = 0;
-                t_u0 = su;
                 t_row0 = 0;
                 t_n = a.T;
                 t_nseg = nseg_s;
                 t_s = 0;
-                su += t_h;
+                sj += gridDim.x;
                 have_tile = true;
                 continue;
             }
@@ -776,23 +797,44 @@ static bool make_weight_maps(CUtensorMap (&m)[FF_HEIGHTS], const void *base, uin
 }
 
 // Expected number of activated experts for T tokens (Eq. N(t): E(1 - (1 - K/E)^T)); the host
-// never sees the routing result, so it sizes the rings from the expected rows per expert.
+// never sees the routing result, so it sizes rings and shared tiles from the expectation.
 static double expected_active_experts(int E, int k, int T)
 {
     return E * (1.0 - pow(1.0 - (double)k / E, (double)T));
 }
 
-// Ring geometry.  While the expected rows per expert are few the pass is a weight stream:
-// 64 KB weight slots (two k boxes of a full tile) and a small token ring.  Near and beyond
-// the ridge the token operand is as large as the weight tile: one k box per slot and a token
-// ring that holds several 128-row entries.
+static int ffn_grid() { return sm_count(); }
+
+// Number of tiles the shared expert's rows are cut into.  A tile is about as tall as the
+// expected per-CTA share of the whole pass, within [min_tile, max_tile] rows: a tensor-core
+// instruction costs the same for any tile height, so tiles below 128 stacked rows (the N
+// operand) would make the pass issue-bound.
+static int shared_tile_count(const moe_config_t &c, int T, int rows_routed, int rows_shared,
+                             int K_routed, int K_shared, int min_tile, int max_tile, int grid)
+{
+    const int nseg_s = (T + FF_SEG - 1) / FF_SEG;
+    const int units = rows_shared >> 4;
+    const double unit_cost = (double)K_shared / K_routed * nseg_s;  // in routed positions
+    const double n_act = expected_active_experts(c.n_experts, c.top_k, T);
+    const double segs_r = n_act * ceil((double)T * c.top_k / n_act / FF_SEG);
+    const double total = units * unit_cost + segs_r * (rows_routed >> 4);
+    int tu = (int)ceil(total / grid / unit_cost);
+    if (tu < (min_tile >> 4))
+        tu = min_tile >> 4;
+    if (tu > (max_tile >> 4))
+        tu = max_tile >> 4;
+    return (units + tu - 1) / tu;
+}
+
+// Ring geometry: one k box per weight slot (32 KB for a full tile); the two boxes of a
+// 128-element k step are issued back to back, so HBM still sees 256 contiguous bytes per
+// row.  The token ring holds at least two entries of the largest segment.
 static void ffn_geometry(const moe_config_t &c, int T, FfnArgs &a)
 {
-    const double per_group = (double)T * c.top_k / expected_active_experts(c.n_experts, c.top_k, T);
-    const bool streaming = per_group <= 48.0;
-    a.kboxes = streaming ? 2 : 1;
+    (void)c;
+    a.kboxes = 1;
     a.w_slot_bytes = 256 * 128 * a.kboxes;  // a full tile: 256 stacked rows per k box
-    const int x_ring_bytes = streaming ? 32 * 1024 : 96 * 1024;
+    const int x_ring_bytes = T > 64 ? 64 * 1024 : 32 * 1024;
     a.x_units = x_ring_bytes / FF_X_UNIT;
     const int avail = FF_SMEM_LIMIT - 1024 - 512;  // alignment slack, static shared memory
     int ns = (avail - x_ring_bytes) / a.w_slot_bytes;
@@ -818,7 +860,7 @@ static cudaError_t launch_ffn(FfnArgs &a, const FfnMaps &maps, cudaStream_t s)
     const size_t smem = (size_t)a.x_units * FF_X_UNIT + (size_t)a.n_w_slots * a.w_slot_bytes + 1024;
     if (a.n_w_slots < 2 || smem > FF_SMEM_LIMIT - 512)
         return cudaErrorInvalidConfiguration;
-    return launch_pdl(ffn_fused_kernel<GATED>, dim3(sm_count()), dim3(FF_THREADS), smem, s, a, maps);
+    return launch_pdl(ffn_fused_kernel<GATED>, dim3(ffn_grid()), dim3(FF_THREADS), smem, s, a, maps);
 }
 
 cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x,
@@ -832,6 +874,9 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
     a.rows[1] = c.shared_inter;
     a.K[0] = a.K[1] = c.hidden;
     a.max_tile = 128;
+    a.shared_tiles = with_shared ? shared_tile_count(c, T, c.inter, c.shared_inter, c.hidden, c.hidden,
+                                                     64, 128, ffn_grid())
+                                 : 0;
     ffn_geometry(c, T, a);
     FfnMaps maps;
     memset(&maps, 0, sizeof maps);
@@ -867,6 +912,9 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
     a.K[0] = c.inter;
     a.K[1] = c.shared_inter;
     a.max_tile = 256;
+    a.shared_tiles = with_shared ? shared_tile_count(c, T, c.hidden, c.hidden, c.inter, c.shared_inter,
+                                                     128, 256, ffn_grid())
+                                 : 0;
     ffn_geometry(c, T, a);
     FfnMaps maps;
     memset(&maps, 0, sizeof maps);
