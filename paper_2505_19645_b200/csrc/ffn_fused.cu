@@ -19,8 +19,10 @@
 // are dealt round-robin to the CTAs; they depend on nothing the layer computes, so they run
 // before the routing result exists, and the routed ranges are then sized so that
 // shared + routed cost is level across the grid.  Inside its range a CTA cuts tiles of at
-// most 128 (gate/up) or 256 (down) rows; for a group with more than 128 token rows it runs
-// the tile once per segment, back to back, so that the second and later passes come from L2.
+// most 128 (gate/up) or 256 (down) rows.  A group with more than 128 token rows has several
+// segments; two segments share one pass over a tile (the weight slot is multiplied with
+// both, one accumulator buffer each), and the shared expert's (tile, segment pair) units are
+// spread over the CTAs so that the units of one tile run at the same time and meet in L2.
 //
 // A weight slot of the shared-memory ring holds `kboxes` 64-element k boxes of one tile
 // (32 KB per box for a full tile), so that one producer/consumer hand-shake moves enough
@@ -66,8 +68,9 @@ struct FfnArgs {
     int32_t *status;
     int T;             // token rows (the shared expert's group)
     int with_shared;   // shared expert present in this launch
-    int shared_tiles;  // tiles of the shared expert's rows, dealt round-robin to the CTAs;
-                       // the first (units % tiles) of them have one 16-row unit more
+    int shared_tiles;  // tiles of the shared expert's rows; (tile, segment pair) units are dealt
+                       // round-robin to the CTAs; the first (units % tiles) tiles have one
+                       // 16-row unit more
     int max_tile;      // weight rows per tile: 128 (gate + up stacked) or 256 (down)
     int kboxes;        // 64-element k boxes per weight slot
     int w_slot_bytes;  // capacity of a weight slot
@@ -232,6 +235,8 @@ __device__ __forceinline__ uint32_t umma_idesc_bf16(int n)
 // ---- kernel ----------------------------------------------------------------------------
 
 // One work item: one segment of token rows of a group against one tile of its weight rows.
+// Two segments of the same group run as a pair on one pass over the tile: the weight slot is
+// loaded once and multiplied with both segments' rows into the two accumulator buffers.
 struct Item {
     int grp;     // 0 routed, 1 shared
     int expert;  // routed expert id (0 for the shared expert)
@@ -239,17 +244,18 @@ struct Item {
     int h;       // weight rows of the tile, multiple of 16
     int row0;    // first token row (sorted row for routed groups, token for the shared expert)
     int n;       // token rows, 1..FF_SEG
+    int role;    // 0 single, 1 first of a pair, 2 second of a pair (shares the first's tile)
 };
 
-// Walks the items of one CTA: its tiles of the shared expert first (they depend on nothing
+// Walks the items of one CTA: its units of the shared expert first (they depend on nothing
 // the layer computes), then its range of the routed groups' rows.  The routed part needs the
 // segment plan, which the preceding kernels write: next() calls griddepcontrol.wait once
 // before it touches the plan (or before reporting the end).
 struct ItemWalk {
     const FfnArgs &a;
     const int max_units;
-    // shared expert: tiles sj, sj + grid, ...
-    int sj, Us, s_base, s_rem, nseg_s;
+    // shared expert: units (tile, segment pair) sj, sj + grid, ... of shared_tiles * pairs_s
+    int sj, Us, s_base, s_rem, nseg_s, pairs_s;
     // routed groups: from (fs, u) to (fs_hi, u_hi); fs = plan index of a group's first segment
     int R0, nseg_total, fs, u, fs_hi, u_hi;
     bool synced, group_loaded;
@@ -257,7 +263,7 @@ struct ItemWalk {
     Segment sg;
     int g_nseg, g_u_end;
     bool have_tile;
-    int t_grp, t_expert, t_u0, t_h, t_row0, t_n, t_nseg, t_s;
+    int t_grp, t_expert, t_u0, t_h, t_row0, t_n, t_s, t_s_end;
 
     __device__ ItemWalk(const FfnArgs &args, bool already_synced)
         : a(args), max_units(args.max_tile >> 4), synced(false), group_loaded(false), have_tile(false)
@@ -267,29 +273,31 @@ struct ItemWalk {
         s_rem = a.shared_tiles ? Us % a.shared_tiles : 0;
         sj = blockIdx.x;
         nseg_s = (a.T + FF_SEG - 1) / FF_SEG;
+        pairs_s = (nseg_s + 1) >> 1;
         R0 = a.rows[0] >> 4;
         nseg_total = fs = u = fs_hi = u_hi = 0;
         if (already_synced)
             sync(false);
     }
-    // First routed position of CTA c.  CTAs [0, r) hold one shared tile more than CTAs [r, G);
+    // First routed position of CTA c.  CTAs [0, r) hold one shared unit more than CTAs [r, G);
     // the routed positions first fill the second class up to the first, the rest is spread
     // over everybody.  Costs are counted in (16 rows x 1 k element x 1 segment): a routed
-    // position costs K[0], a shared unit K[1] * nseg_s.  Integer arithmetic only, so every
-    // role of every CTA derives the same bounds.
+    // position costs K[0], a shared unit (tile height) * K[1] * (segments per unit).  Integer
+    // arithmetic only, so every role of every CTA derives the same bounds.
     __device__ long long routed_bound(int c, long long P) const
     {
         const int G = gridDim.x;
-        const int r = a.shared_tiles % G;
+        const int r = (a.shared_tiles * pairs_s) % G;
         if (r == 0)
             return P * c / G;
-        const long long tile_cost = (long long)(s_base + (s_rem ? 1 : 0)) * a.K[1] * nseg_s;
+        const long long unit_cost =
+            (long long)(s_base + (s_rem ? 1 : 0)) * a.K[1] * nseg_s / pairs_s;
         const long long p_cost = P * a.K[0];
         const int n_lo = G - r;
-        if (p_cost <= tile_cost * n_lo)
+        if (p_cost <= unit_cost * n_lo)
             return c < r ? 0 : P * (c - r) / n_lo;
-        const long long extra = p_cost - tile_cost * n_lo;  // spread over all G CTAs
-        return (extra * c + tile_cost * G * (c > r ? c - r : 0)) / ((long long)G * a.K[0]);
+        const long long extra = p_cost - unit_cost * n_lo;  // spread over all G CTAs
+        return (extra * c + unit_cost * G * (c > r ? c - r : 0)) / ((long long)G * a.K[0]);
     }
     // position p (in units of 16 rows x one segment, groups laid end to end, each group's
     // units repeated for all its segments) -> (group, row unit)
@@ -320,27 +328,30 @@ struct ItemWalk {
     {
         for (;;) {
             if (have_tile) {
-                if (t_s < t_nseg) {
+                if (t_s < t_s_end) {
                     it.grp = t_grp;
                     it.expert = t_expert;
                     it.f0 = t_u0 << 4;
                     it.h = t_h << 4;
                     it.row0 = t_row0 + t_s * FF_SEG;
                     it.n = min(FF_SEG, t_n - t_s * FF_SEG);
+                    // segments 2q and 2q+1 of a tile form a pair
+                    it.role = (t_s & 1) ? 2 : (t_s + 1 < t_s_end ? 1 : 0);
                     ++t_s;
                     return true;
                 }
                 have_tile = false;
             }
-            if (sj < a.shared_tiles) {  // next tile of the shared expert
-                t_u0 = sj * s_base + min(sj, s_rem);
-                t_h = s_base + (sj < s_rem ? 1 : 0);
+            if (sj < a.shared_tiles * pairs_s) {  // next unit of the shared expert
+                const int tile = sj / pairs_s, q = sj - tile * pairs_s;
+                t_u0 = tile * s_base + min(tile, s_rem);
+                t_h = s_base + (tile < s_rem ? 1 : 0);
                 t_grp = 1;
                 t_expert = 0;
                 t_row0 = 0;
                 t_n = a.T;
-                t_nseg = nseg_s;
-                t_s = 0;
+                t_s = 2 * q;
+                t_s_end = min(nseg_s, 2 * q + 2);
                 sj += gridDim.x;
                 have_tile = true;
                 continue;
@@ -355,15 +366,15 @@ struct ItemWalk {
                 g_u_end = fs == fs_hi ? u_hi : R0;
                 group_loaded = true;
             }
-            if (u < g_u_end) {  // next tile of this group
+            if (u < g_u_end) {  // next tile of this group, all its segments
                 t_h = min(max_units, g_u_end - u);
                 t_grp = 0;
                 t_expert = sg.expert;
                 t_u0 = u;
                 t_row0 = sg.row0;
                 t_n = sg.n;
-                t_nseg = g_nseg;
                 t_s = 0;
+                t_s_end = g_nseg;
                 u += t_h;
                 have_tile = true;
                 continue;
@@ -494,6 +505,8 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                     griddep_launch();  // after the wait: dependents may rely on the plan
                     launched = true;
                 }
+                if (it.role == 2)
+                    continue;  // rides on the tile loaded for the first of its pair
                 const int K = args.K[it.grp];
                 const uint32_t tile_bytes = (uint32_t)it.h * 128u;
                 const int wrow = it.expert * args.rows[0] + it.f0;  // expert = 0 for the shared kind
@@ -552,40 +565,48 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             bool ok = true;
             Item it;
             while (ok && walk.next(it)) {
+                // a pair alternates its two segments' entries, k step by k step
+                Item it2 = it;
+                const int nsub = it.role == 1 ? 2 : 1;
+                if (nsub == 2 && !walk.next(it2))
+                    break;  // cannot happen: a first is always followed by its second
                 const CUtensorMap *mx = &maps.x[it.grp];
                 const int K = args.K[it.grp];
-                const int pieces = pieces16(it.n);
-                const int m = pieces * kb;
-                for (int k0 = 0; k0 < K; k0 += 64 * kb) {
+                for (int k0 = 0; ok && k0 < K; k0 += 64 * kb) {
                     const int nbox = min(kb, (K - k0 + 63) >> 6);
-                    const int j = ring.count;
-                    int pad;
-                    const int at = ring.place(m, pad);
-                    const int v_end = v_cur + pad + m;
-                    // the entry's units (and its barrier pair) must have been released
-                    // (with nothing outstanding the whole ring is free, padding included)
-                    while (released < j &&
-                           (j - released >= FF_X_ENTRIES || v_end - v_rel > args.x_units)) {
-                        const int r = released % FF_X_ENTRIES;
-                        if (!mbar_wait(x_empty(r), (uint32_t)(released / FF_X_ENTRIES) & 1u, abortp,
-                                       args.status)) {
-                            ok = false;
-                            break;
+                    for (int sub = 0; sub < nsub; ++sub) {
+                        const Item &cur = sub ? it2 : it;
+                        const int pieces = pieces16(cur.n);
+                        const int m = pieces * kb;
+                        const int j = ring.count;
+                        int pad;
+                        const int at = ring.place(m, pad);
+                        const int v_end = v_cur + pad + m;
+                        // the entry's units (and its barrier pair) must have been released
+                        // (with nothing outstanding the whole ring is free, padding included)
+                        while (released < j &&
+                               (j - released >= FF_X_ENTRIES || v_end - v_rel > args.x_units)) {
+                            const int r = released % FF_X_ENTRIES;
+                            if (!mbar_wait(x_empty(r), (uint32_t)(released / FF_X_ENTRIES) & 1u, abortp,
+                                           args.status)) {
+                                ok = false;
+                                break;
+                            }
+                            v_rel = v_end_of[r];
+                            ++released;
                         }
-                        v_rel = v_end_of[r];
-                        ++released;
+                        if (!ok)
+                            break;
+                        const int e = j % FF_X_ENTRIES;
+                        v_end_of[e] = v_end;
+                        v_cur = v_end;
+                        const uint32_t base = ring_x + (uint32_t)at * FF_X_UNIT;
+                        mbar_expect_tx(x_full(e), (uint32_t)(nbox * pieces) * FF_X_UNIT);
+                        for (int b = 0; b < nbox; ++b)
+                            for (int p = 0; p < pieces; ++p)
+                                tma_load_2d(base + (uint32_t)(b * pieces + p) * FF_X_UNIT, mx, x_full(e),
+                                            k0 + 64 * b, cur.row0 + 16 * p);
                     }
-                    if (!ok)
-                        break;
-                    const int e = j % FF_X_ENTRIES;
-                    v_end_of[e] = v_end;
-                    v_cur = v_end;
-                    const uint32_t base = ring_x + (uint32_t)at * FF_X_UNIT;
-                    mbar_expect_tx(x_full(e), (uint32_t)(nbox * pieces) * FF_X_UNIT);
-                    for (int b = 0; b < nbox; ++b)
-                        for (int p = 0; p < pieces; ++p)
-                            tma_load_2d(base + (uint32_t)(b * pieces + p) * FF_X_UNIT, mx, x_full(e),
-                                        k0 + 64 * b, it.row0 + 16 * p);
                 }
             }
             if (!walk.synced)
@@ -607,49 +628,68 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             int n_items = 0;
             Item it;
             while (ok && walk.next(it)) {
-                const int buf = n_items & 1;
-                const uint32_t acc_phase = (uint32_t)(n_items >> 1) & 1u;
-                ++n_items;
-                if (!mbar_wait(acc_empty(buf), acc_phase ^ 1u, abortp, args.status))
+                Item it2 = it;
+                const int nsub = it.role == 1 ? 2 : 1;
+                if (nsub == 2 && !walk.next(it2))
+                    break;  // cannot happen: a first is always followed by its second
+                int buf[2];
+                for (int sub = 0; ok && sub < nsub; ++sub) {
+                    buf[sub] = n_items & 1;
+                    const uint32_t acc_phase = (uint32_t)(n_items >> 1) & 1u;
+                    ++n_items;
+                    if (!mbar_wait(acc_empty(buf[sub]), acc_phase ^ 1u, abortp, args.status))
+                        ok = false;
+                }
+                if (!ok)
                     break;
                 tc_fence_after();
                 const uint32_t tile_bytes = (uint32_t)it.h * 128u;
                 const uint32_t idesc = umma_idesc_bf16(NW * it.h);
-                const uint32_t d0 = tmem_base + (uint32_t)(buf * ACC_COLS);
                 const int K = args.K[it.grp];
-                const int pieces = pieces16(it.n);
-                const int m = pieces * kb;
-                for (int k0 = 0; k0 < K; k0 += 64 * kb) {
+                for (int k0 = 0; ok && k0 < K; k0 += 64 * kb) {
                     const int nbox = min(kb, (K - k0 + 63) >> 6);
-                    const int j = ring.count;
-                    int pad;
-                    const int at = ring.place(m, pad);
-                    const int e = j % FF_X_ENTRIES;
-                    if (!mbar_wait(x_full(e), (uint32_t)(j / FF_X_ENTRIES) & 1u, abortp, args.status) ||
-                        !mbar_wait(w_full(sw), pw, abortp, args.status)) {
+                    // the weight slot is multiplied with one or two segments' token entries
+                    uint32_t xbase[2];
+                    int xe[2], pieces[2];
+                    for (int sub = 0; sub < nsub; ++sub) {
+                        pieces[sub] = pieces16(sub ? it2.n : it.n);
+                        const int j = ring.count;
+                        int pad;
+                        const int at = ring.place(pieces[sub] * kb, pad);
+                        xe[sub] = j % FF_X_ENTRIES;
+                        xbase[sub] = ring_x + (uint32_t)at * FF_X_UNIT;
+                        if (!mbar_wait(x_full(xe[sub]), (uint32_t)(j / FF_X_ENTRIES) & 1u, abortp,
+                                       args.status))
+                            ok = false;
+                    }
+                    if (!ok || !mbar_wait(w_full(sw), pw, abortp, args.status)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t xbase = ring_x + (uint32_t)at * FF_X_UNIT;
                     const uint32_t wbase = ring_w + sw * args.w_slot_bytes;
-                    for (int b = 0; b < nbox; ++b) {
+                    for (int sub = 0; sub < nsub; ++sub) {
+                        const uint32_t d0 = tmem_base + (uint32_t)(buf[sub] * ACC_COLS);
+                        for (int b = 0; b < nbox; ++b) {
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const uint32_t accum = (k0 | b | q) != 0 ? 1u : 0u;
-                            umma_bf16(d0, umma_desc_sw128(xbase + (uint32_t)(b * pieces) * FF_X_UNIT + q * 32),
-                                      umma_desc_sw128(wbase + b * NW * tile_bytes + q * 32), idesc, accum);
+                            for (int q = 0; q < 4; ++q) {
+                                const uint32_t accum = (k0 | b | q) != 0 ? 1u : 0u;
+                                umma_bf16(d0,
+                                          umma_desc_sw128(xbase[sub] + (uint32_t)(b * pieces[sub]) * FF_X_UNIT + q * 32),
+                                          umma_desc_sw128(wbase + b * NW * tile_bytes + q * 32), idesc, accum);
+                            }
                         }
+                        umma_commit(x_empty(xe[sub]));
                     }
-                    umma_commit(w_empty(sw));  // reusable once these MMAs have read them
-                    umma_commit(x_empty(e));
+                    umma_commit(w_empty(sw));  // reusable once these MMAs have read it
                     if (++sw == NS) {
                         sw = 0;
                         pw ^= 1u;
                     }
                 }
                 if (ok)
-                    umma_commit(acc_full(buf));  // accumulator complete
+                    for (int sub = 0; sub < nsub; ++sub)
+                        umma_commit(acc_full(buf[sub]));  // accumulators complete
             }
             if (!walk.synced)
                 walk.sync(true);
@@ -805,20 +845,22 @@ static double expected_active_experts(int E, int k, int T)
 
 static int ffn_grid() { return sm_count(); }
 
-// Number of tiles the shared expert's rows are cut into.  A tile is about as tall as the
-// expected per-CTA share of the whole pass, within [min_tile, max_tile] rows: a tensor-core
+// Number of tiles the shared expert's rows are cut into.  The shared expert's work units are
+// (tile, segment pair); a unit should cost about the expected per-CTA share of the whole pass
+// (or less), with the tile height within [min_tile, max_tile] rows: a tensor-core
 // instruction costs the same for any tile height, so tiles below 128 stacked rows (the N
 // operand) would make the pass issue-bound.
 static int shared_tile_count(const moe_config_t &c, int T, int rows_routed, int rows_shared,
                              int K_routed, int K_shared, int min_tile, int max_tile, int grid)
 {
     const int nseg_s = (T + FF_SEG - 1) / FF_SEG;
+    const int pairs_s = (nseg_s + 1) / 2;
     const int units = rows_shared >> 4;
-    const double unit_cost = (double)K_shared / K_routed * nseg_s;  // in routed positions
+    const double k_ratio = (double)K_shared / K_routed;  // cost of a shared row unit per segment
     const double n_act = expected_active_experts(c.n_experts, c.top_k, T);
     const double segs_r = n_act * ceil((double)T * c.top_k / n_act / FF_SEG);
-    const double total = units * unit_cost + segs_r * (rows_routed >> 4);
-    int tu = (int)ceil(total / grid / unit_cost);
+    const double total = units * k_ratio * nseg_s + segs_r * (rows_routed >> 4);
+    int tu = (int)ceil(total / grid / (k_ratio * nseg_s / pairs_s));
     if (tu < (min_tile >> 4))
         tu = min_tile >> 4;
     if (tu > (max_tile >> 4))
