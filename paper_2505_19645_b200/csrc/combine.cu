@@ -13,6 +13,8 @@ combine_kernel(const __nv_bfloat16 *__restrict__ y, const int32_t *__restrict__ 
                const float *__restrict__ shared_scale, int T, int H, int k,
                __nv_bfloat16 *__restrict__ out)
 {
+    griddep_launch();
+    griddep_wait();  // y and shared_y come from the preceding kernel
     const int vec_per_row = H >> 3;
     const size_t total = (size_t)T * vec_per_row;
     for (size_t i = blockIdx.x * (size_t)CB_THREADS + threadIdx.x; i < total;
@@ -71,9 +73,8 @@ cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, const 
     const size_t cap = (size_t)sm_count() * 8;
     if (blocks > cap)
         blocks = cap;
-    combine_kernel<<<(unsigned)blocks, CB_THREADS, 0, s>>>(y, inv_perm, topk_w, shared_y,
-                                                          shared_scale, T, c.hidden, c.top_k, out);
-    return cudaGetLastError();
+    return launch_pdl(combine_kernel, dim3((unsigned)blocks), dim3(CB_THREADS), 0, s, y, inv_perm,
+                      topk_w, shared_y, shared_scale, T, c.hidden, c.top_k, out);
 }
 
 }  // namespace moe

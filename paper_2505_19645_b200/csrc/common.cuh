@@ -170,6 +170,18 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Programmatic dependent launch.  Every kernel of the layer is launched with launch_pdl and
+// follows one discipline: it executes griddep_wait() before it reads or writes anything that
+// a kernel of the same layer call produces or consumes, and before it exits; the first kernel
+// of a call (router logits) and the gate/up pass trigger their dependents only after their
+// own wait, so whatever a later kernel touches before ITS wait (the caller's inputs only) is
+// older than the call itself.
+// Blocks until the preceding kernel in the stream has completed and its writes are visible
+// (returns at once when the kernel was not launched as a programmatic dependent).
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel in the stream start its own prologue.
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // 128-bit streaming load: weights are read exactly once, keep them out of L1.
 __device__ __forceinline__ uint4 ld_stream_v4(const void *p)
 {

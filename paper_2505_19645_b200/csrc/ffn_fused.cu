@@ -24,9 +24,9 @@
 // both, one accumulator buffer each), and the shared expert's (tile, segment pair) units are
 // spread over the CTAs so that the units of one tile run at the same time and meet in L2.
 //
-// A weight slot of the shared-memory ring holds `kboxes` 64-element k boxes of one tile
-// (32 KB per box for a full tile), so that one producer/consumer hand-shake moves enough
-// bytes to keep HBM busy; the token operand lives in a second ring whose entries are sized
+// A weight slot of the shared-memory ring holds two 64-element k boxes of one tile (64 KB
+// for a full tile), so that one producer/consumer hand-shake moves enough bytes to keep HBM
+// busy and every weight row is requested in 256 contiguous bytes; the token operand lives in a second ring whose entries are sized
 // by the segment's row count.
 //
 // CTA = 7 warps.  warp 0: weight producer (one lane issues TMA), warp 1: MMA issuer (one
@@ -168,12 +168,6 @@ __device__ __forceinline__ void prefetch_map(const CUtensorMap *map)
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// Blocks until the preceding kernel in the stream has completed and its writes are visible
-// (returns at once when the kernel was not launched as a programmatic dependent).
-__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-// Lets the next kernel in the stream start its own prologue.
-__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
                                           uint32_t idesc, uint32_t accumulate)
@@ -868,15 +862,15 @@ static int shared_tile_count(const moe_config_t &c, int T, int rows_routed, int 
     return (units + tu - 1) / tu;
 }
 
-// Ring geometry: one k box per weight slot (32 KB for a full tile); the two boxes of a
-// 128-element k step are issued back to back, so HBM still sees 256 contiguous bytes per
-// row.  The token ring holds at least two entries of the largest segment.
-static void ffn_geometry(const moe_config_t &c, int T, FfnArgs &a)
+// Ring geometry: two k boxes per weight slot (64 KB for a full tile: every row is fetched in
+// 256 contiguous bytes, which both HBM and L2 serve markedly faster than 128).  The token
+// ring holds two entries of the largest possible segment while no group can exceed 64 rows,
+// three 128-row entries otherwise (a pair of segments needs two at once).
+static void ffn_geometry(int T, FfnArgs &a)
 {
-    (void)c;
-    a.kboxes = 1;
+    a.kboxes = 2;
     a.w_slot_bytes = 256 * 128 * a.kboxes;  // a full tile: 256 stacked rows per k box
-    const int x_ring_bytes = T > 64 ? 64 * 1024 : 32 * 1024;
+    const int x_ring_bytes = T > 64 ? 96 * 1024 : 32 * 1024;
     a.x_units = x_ring_bytes / FF_X_UNIT;
     const int avail = FF_SMEM_LIMIT - 1024 - 512;  // alignment slack, static shared memory
     int ns = (avail - x_ring_bytes) / a.w_slot_bytes;
@@ -919,7 +913,7 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
     a.shared_tiles = with_shared ? shared_tile_count(c, T, c.inter, c.shared_inter, c.hidden, c.hidden,
                                                      64, 128, ffn_grid())
                                  : 0;
-    ffn_geometry(c, T, a);
+    ffn_geometry(T, a);
     FfnMaps maps;
     memset(&maps, 0, sizeof maps);
     bool ok = make_weight_maps(maps.w[0][0], w.w_gate, E * c.inter, H) &&
@@ -957,7 +951,7 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
     a.shared_tiles = with_shared ? shared_tile_count(c, T, c.hidden, c.hidden, c.inter, c.shared_inter,
                                                      128, 256, ffn_grid())
                                  : 0;
-    ffn_geometry(c, T, a);
+    ffn_geometry(T, a);
     FfnMaps maps;
     memset(&maps, 0, sizeof maps);
     bool ok = make_weight_maps(maps.w[0][0], w.w_down, E * H, c.inter) &&

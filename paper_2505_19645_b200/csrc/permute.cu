@@ -78,9 +78,11 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
     __shared__ int flag[MOE_MAX_EXPERTS];
     __shared__ int tmp[MOE_MAX_EXPERTS];
     __shared__ int total;
+    griddep_launch();
     const int tid = threadIdx.x;
     if (tid < MOE_MAX_EXPERTS)
         hist[tid] = 0;
+    griddep_wait();  // the expert indices come from the preceding kernel
     __syncthreads();
     for (int a = tid; a < A; a += PERM_THREADS) {
         const int e = topk_idx[a];
@@ -152,9 +154,8 @@ cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int
     PlanView pv{};
     if (plan)
         pv = *plan;
-    permute_kernel<<<blocks, PERM_THREADS, 0, s>>>(idx, T * c.top_k, E, counts, offsets, perm,
-                                                   inv_perm, active, n_active, status, pv);
-    return cudaGetLastError();
+    return launch_pdl(permute_kernel, dim3(blocks), dim3(PERM_THREADS), 0, s, idx, T * c.top_k, E,
+                      counts, offsets, perm, inv_perm, active, n_active, status, pv);
 }
 
 // Stand-alone plan (moe_grouped_swiglu gets its offsets from the caller).
@@ -166,6 +167,8 @@ plan_kernel(const int32_t *__restrict__ offsets, int E, int32_t *__restrict__ st
     __shared__ int scan[MOE_MAX_EXPERTS];
     __shared__ int tmp[MOE_MAX_EXPERTS];
     __shared__ int total;
+    griddep_wait();
+    griddep_launch();
     const int tid = threadIdx.x;
     int row0 = 0, n = 0;
     if (tid < E) {
@@ -182,8 +185,8 @@ cudaError_t launch_plan(const moe_config_t &c, int T, const int32_t *offsets, in
                         PlanView plan, cudaStream_t s)
 {
     (void)T;
-    plan_kernel<<<1, MOE_MAX_EXPERTS, 0, s>>>(offsets, c.n_experts, status, plan);
-    return cudaGetLastError();
+    return launch_pdl(plan_kernel, dim3(1), dim3(MOE_MAX_EXPERTS), 0, s, offsets, c.n_experts, status,
+                      plan);
 }
 
 }  // namespace moe

@@ -18,6 +18,8 @@ route_topk_kernel(const float *__restrict__ logits, int T, int E, int k, int sco
                   int renormalize, float routed_scale, int32_t *__restrict__ topk_idx,
                   float *__restrict__ topk_w)
 {
+    griddep_launch();
+    griddep_wait();  // the logits come from the preceding kernel
     const int lane = threadIdx.x & 31;
     const int t = (int)((blockIdx.x * (size_t)blockDim.x + threadIdx.x) >> 5);
     if (t >= T)
@@ -104,8 +106,9 @@ cudaError_t launch_route_topk(const moe_config_t &c, const float *logits, int T,
     const int threads = 128;
     const int blocks = (int)(((size_t)T * 32 + threads - 1) / threads);
 #define MOE_TOPK_LAUNCH(V)                                                                     \
-    route_topk_kernel<V><<<blocks, threads, 0, s>>>(logits, T, E, c.top_k, c.score_fn,        \
-                                                   c.renormalize, c.routed_scale, idx, wts)
+    err = launch_pdl(route_topk_kernel<V>, dim3(blocks), dim3(threads), 0, s, logits, T, E,    \
+                     c.top_k, c.score_fn, c.renormalize, c.routed_scale, idx, wts)
+    cudaError_t err = cudaSuccess;
     if (E <= 32)
         MOE_TOPK_LAUNCH(1);
     else if (E <= 64)
@@ -117,7 +120,7 @@ cudaError_t launch_route_topk(const moe_config_t &c, const float *logits, int T,
     else
         MOE_TOPK_LAUNCH(16);
 #undef MOE_TOPK_LAUNCH
-    return cudaGetLastError();
+    return err;
 }
 
 }  // namespace moe

@@ -66,6 +66,8 @@ router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restric
                      float *__restrict__ shared_scale)
 {
     __shared__ float part[RL_WARPS][NCH][4][32];
+    griddep_wait();    // first kernel of a layer call: everything older is complete from here on
+    griddep_launch();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;
     const int e0 = blockIdx.x * 16;
@@ -160,9 +162,9 @@ cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
     dim3 grid(e_tiles, (T + 8 * nch - 1) / (8 * nch));
     const __nv_bfloat16 *w_sg = static_cast<const __nv_bfloat16 *>(w.w_shared_gate);
 #define MOE_RL_LAUNCH(N)                                                                    \
-    router_logits_kernel<N><<<grid, RL_WARPS * 32, 0, s>>>(x, w.w_router, w.router_bias, w_sg, T, \
-                                                          c.hidden, c.n_experts, n_rows, logits, \
-                                                          shared_scale)
+    err = launch_pdl(router_logits_kernel<N>, grid, dim3(RL_WARPS * 32), 0, s, x, w.w_router,    \
+                     w.router_bias, w_sg, T, c.hidden, c.n_experts, n_rows, logits, shared_scale)
+    cudaError_t err = cudaSuccess;
     switch (nch) {
     case 1: MOE_RL_LAUNCH(1); break;
     case 2: MOE_RL_LAUNCH(2); break;
@@ -170,7 +172,7 @@ cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
     default: MOE_RL_LAUNCH(8); break;
     }
 #undef MOE_RL_LAUNCH
-    return cudaGetLastError();
+    return err;
 }
 
 }  // namespace moe
