@@ -30,6 +30,9 @@ from paper_2505_19645_b200 import replicas, workloads as wl  # noqa: E402
 L2_FLUSH_BYTES = 512 << 20
 DEFAULT_CONFIG = "qwen1.5-moe-a2.7b"
 DEFAULT_B, DEFAULT_GAMMA = 32, 3
+# dram__bytes_read.sum + dram__bytes_write.sum of one gate/up launch on the default workload
+# (profiles/ffn_fused_qwen15_T128.md); set to None whenever that kernel changes
+NCU_GATE_UP_DRAM_BYTES = 749098752 + 10349312
 
 
 def load_peaks():
@@ -344,8 +347,13 @@ def main():
         achieved = gu_flops / (k_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],
                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"]}
-    roofline.update({"traffic": None, "kernel": "gate/up + SwiGLU", "kernel_ms": k_ms,
-                     "algorithmic_bytes": gu_bytes, "peak_source": peaks["source"]})
+    # DRAM bytes of one launch from the ncu capture summarised in profiles/ (taken on the
+    # default workload; it scales with the activated bytes, so other workloads report null)
+    traffic = NCU_GATE_UP_DRAM_BYTES if (args.config, B, gamma, args.zipf) == (
+        DEFAULT_CONFIG, DEFAULT_B, DEFAULT_GAMMA, None) else None
+    roofline.update({"traffic": traffic, "kernel": "ffn_fused_kernel<gate/up + SwiGLU>",
+                     "kernel_ms": k_ms, "algorithmic_bytes": gu_bytes,
+                     "peak_source": peaks["source"]})
 
     # whole-layer roofline: slower of activated-expert bytes over HBM and flops at tensor peak
     def layer_roof_ms(Tn, nact):
