@@ -161,6 +161,34 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+// The same load with an L2 eviction-priority policy (see createpolicy below).
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                                 int c0, int c1, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%3, %4}], [%2], %5;"
+        :
+        : "r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "l"(policy)
+        : "memory");
+}
+
+// L2 policies: weights that are read once should leave L2 first, the token rows (re-read for
+// every weight tile of their group) last -- otherwise the weight stream, which is larger than
+// L2, evicts them between two tiles.
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
 __device__ __forceinline__ void prefetch_map(const CUtensorMap *map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
@@ -239,6 +267,7 @@ struct Item {
     int row0;    // first token row (sorted row for routed groups, token for the shared expert)
     int n;       // token rows, 1..FF_SEG
     int role;    // 0 single, 1 first of a pair, 2 second of a pair (shares the first's tile)
+    int w_once;  // the tile's weights are read by this item (or pair) only
 };
 
 // Walks the items of one CTA: its units of the shared expert first (they depend on nothing
@@ -331,6 +360,7 @@ struct ItemWalk {
                     it.n = min(FF_SEG, t_n - t_s * FF_SEG);
                     // segments 2q and 2q+1 of a tile form a pair
                     it.role = (t_s & 1) ? 2 : (t_s + 1 < t_s_end ? 1 : 0);
+                    it.w_once = t_grp == 0 ? (t_s_end <= 2) : (nseg_s <= 2);
                     ++t_s;
                     return true;
                 }
@@ -487,6 +517,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             // items run before the wait.  Down pass: every weight tile may be fetched ahead --
             // the launch order guarantees that the plan is complete when this kernel starts.
             ItemWalk walk(args, !GATED);
+            const uint64_t pol_once = l2_policy_evict_first();
             bool launched = !GATED;
             if (!GATED)
                 griddep_launch();
@@ -521,7 +552,11 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                             while (rem > 0) {
                                 const int hi = rem >= 128 ? 0 : (rem >= 64 ? 1 : (rem >= 32 ? 2 : 3));
                                 const int bh = 128 >> hi;
-                                tma_load_2d(dst, &maps.w[it.grp][m][hi], w_full(slot), k0 + 64 * b, row);
+                                if (it.w_once)
+                                    tma_load_2d_hint(dst, &maps.w[it.grp][m][hi], w_full(slot), k0 + 64 * b,
+                                                     row, pol_once);
+                                else
+                                    tma_load_2d(dst, &maps.w[it.grp][m][hi], w_full(slot), k0 + 64 * b, row);
                                 dst += (uint32_t)bh * 128u;
                                 row += bh;
                                 rem -= bh;
@@ -553,6 +588,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 griddep_wait();
             ItemWalk walk(args, !GATED);
             XRingWalk ring(args.x_units);
+            const uint64_t pol_keep = l2_policy_evict_last();
             int released = 0;          // entries known to have been consumed
             int v_cur = 0, v_rel = 0;  // virtual unit positions: issued up to / released up to
             int v_end_of[FF_X_ENTRIES];
@@ -598,8 +634,8 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                         mbar_expect_tx(x_full(e), (uint32_t)(nbox * pieces) * FF_X_UNIT);
                         for (int b = 0; b < nbox; ++b)
                             for (int p = 0; p < pieces; ++p)
-                                tma_load_2d(base + (uint32_t)(b * pieces + p) * FF_X_UNIT, mx, x_full(e),
-                                            k0 + 64 * b, cur.row0 + 16 * p);
+                                tma_load_2d_hint(base + (uint32_t)(b * pieces + p) * FF_X_UNIT, mx, x_full(e),
+                                                 k0 + 64 * b, cur.row0 + 16 * p, pol_keep);
                     }
                 }
             }
