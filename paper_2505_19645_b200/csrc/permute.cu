@@ -7,27 +7,43 @@ namespace moe {
 constexpr int PERM_THREADS = 1024;  // 32 warps: one warp places one expert
 
 // Exclusive scan of vals[0..n) (n <= MOE_MAX_EXPERTS <= blockDim.x) in shared memory;
-// returns the total in *total.  All threads of the block must call it.
+// returns the total in *total.  All threads of the block must call it.  Warp shuffles inside
+// each group of 32 entries, then one warp scans the 16 group sums (tmp).
 __device__ void block_exclusive_scan(int *vals, int *tmp, int n, int *total)
 {
-    const int tid = threadIdx.x;
-    int v = tid < n ? vals[tid] : 0;
-    if (tid < MOE_MAX_EXPERTS)
-        tmp[tid] = v;
-    __syncthreads();
-    for (int off = 1; off < MOE_MAX_EXPERTS; off <<= 1) {
-        int add = 0;
-        if (tid < MOE_MAX_EXPERTS && tid >= off)
-            add = tmp[tid - off];
-        __syncthreads();
-        if (tid < MOE_MAX_EXPERTS)
-            tmp[tid] += add;
-        __syncthreads();
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    constexpr int NW = MOE_MAX_EXPERTS / 32;
+    int v = 0, incl = 0;
+    if (wid < NW) {
+        v = tid < n ? vals[tid] : 0;
+        incl = v;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off)
+                incl += o;
+        }
+        if (lane == 31)
+            tmp[wid] = incl;
     }
-    if (tid < n)
-        vals[tid] = tmp[tid] - v;  // inclusive -> exclusive
-    if (tid == 0)
-        *total = tmp[MOE_MAX_EXPERTS - 1];
+    __syncthreads();
+    if (wid == 0) {
+        const int w = lane < NW ? tmp[lane] : 0;
+        int wi = w;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, wi, off);
+            if (lane >= off)
+                wi += o;
+        }
+        if (lane < NW)
+            tmp[lane] = wi - w;  // exclusive offset of each group
+        if (lane == NW - 1)
+            *total = wi;
+    }
+    __syncthreads();
+    if (wid < NW && tid < n)
+        vals[tid] = tmp[wid] + incl - v;
     __syncthreads();
 }
 

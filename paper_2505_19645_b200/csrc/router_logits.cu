@@ -4,13 +4,14 @@
 // The fp32 router row is split on the fly into three bf16 terms  w = hi + mid + lo  (each
 // remainder is exact in fp32, so the three terms carry 24 mantissa bits), the bf16 token
 // values are exact, and the three partial products are accumulated in fp32 by
-// m16n8k16 MMAs.  A CTA owns 16 router rows x (8*NCH) tokens; its 8 warps split H and are
+// m16n8k16 MMAs.  A CTA owns 16 router rows x (8*NCH) tokens; its 16 warps split H and are
 // summed through shared memory, so even T = 1 keeps every load short and parallel.
 #include "common.cuh"
 
 namespace moe {
 
-constexpr int RL_WARPS = 8;
+// warps per CTA (they split H): 16 for the small token tiles that latency-bound calls use
+#define RL_WARPS_FOR(nch) ((nch) <= 2 ? 16 : 8)
 
 struct Split3 {
     uint32_t hi, mid, lo;  // two bf16 each
@@ -59,12 +60,13 @@ __device__ __forceinline__ void load_row8(const RowSrc &r, int k, float (&v)[8])
 }
 
 template <int NCH>
-__global__ void __launch_bounds__(RL_WARPS * 32)
+__global__ void __launch_bounds__(RL_WARPS_FOR(NCH) * 32)
 router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ w_router,
                      const float *__restrict__ bias, const __nv_bfloat16 *__restrict__ w_sg,
                      int T, int H, int E, int n_rows, float *__restrict__ logits,
                      float *__restrict__ shared_scale)
 {
+    constexpr int RL_WARPS = RL_WARPS_FOR(NCH);
     __shared__ float part[RL_WARPS][NCH][4][32];
     griddep_wait();    // first kernel of a layer call: everything older is complete from here on
     griddep_launch();
@@ -96,7 +98,7 @@ router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restric
 
     const int nsteps = H >> 5;
     const int s0 = warp * nsteps / RL_WARPS, s1 = (warp + 1) * nsteps / RL_WARPS;
-#pragma unroll 2
+#pragma unroll 4
     for (int s = s0; s < s1; ++s) {
         const int k = s * 32;
         float lo8[8], hi8[8];
@@ -162,7 +164,7 @@ cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
     dim3 grid(e_tiles, (T + 8 * nch - 1) / (8 * nch));
     const __nv_bfloat16 *w_sg = static_cast<const __nv_bfloat16 *>(w.w_shared_gate);
 #define MOE_RL_LAUNCH(N)                                                                    \
-    err = launch_pdl(router_logits_kernel<N>, grid, dim3(RL_WARPS * 32), 0, s, x, w.w_router,    \
+    err = launch_pdl(router_logits_kernel<N>, grid, dim3(RL_WARPS_FOR(N) * 32), 0, s, x, w.w_router,    \
                      w.router_bias, w_sg, T, c.hidden, c.n_experts, n_rows, logits, shared_scale)
     cudaError_t err = cudaSuccess;
     switch (nch) {
