@@ -132,7 +132,8 @@ static thread_local bool g_probe_armed = false;  // only moe_verify_layer arms i
 PlanView plan_view(char *ws, const Workspace &L)
 {
     return PlanView{reinterpret_cast<int32_t *>(ws + L.plan_header),
-                    reinterpret_cast<Segment *>(ws + L.plan_seg)};
+                    reinterpret_cast<Segment *>(ws + L.plan_seg),
+                    reinterpret_cast<int32_t *>(ws + L.plan_pairs)};
 }
 
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,

@@ -26,10 +26,12 @@ struct Segment {
     int32_t first_seg;  // plan index of the group's first segment
 };
 
-// plan header (ints): [0] number of segments over all activated experts
+// plan header (ints): [0] number of segments over all activated experts,
+//                     [1] number of segment pairs (segments 2q and 2q+1 of a group form a pair)
 struct PlanView {
     int32_t *header;
-    Segment *seg;  // capacity max_segments()
+    Segment *seg;         // capacity max_segments()
+    int32_t *pair_first;  // plan index of every pair's first segment, capacity max_segments()
 };
 
 __host__ __device__ inline int max_segments(int E, int A) { return E + A / SEG_TOKENS + 1; }
@@ -51,6 +53,7 @@ struct Workspace {
     size_t inv_perm;      // i32 [A]
     size_t plan_header;   // i32 [PLAN_HEADER_INTS]
     size_t plan_seg;      // Segment[max_segments]
+    size_t plan_pairs;    // i32 [max_segments]
     size_t x_sorted;      // bf16 [A, H]      token rows in sorted order
     size_t h;             // bf16 [A, I]      SwiGLU intermediate, sorted order
     size_t h_shared;      // bf16 [T, I_s]
@@ -84,6 +87,7 @@ inline Workspace workspace_layout(const moe_config_t &c, int T)
     w.inv_perm = take(A * 4);
     w.plan_header = take(PLAN_HEADER_INTS * 4);
     w.plan_seg = take(sizeof(Segment) * (size_t)max_segments((int)E, (int)A));
+    w.plan_pairs = take(4 * (size_t)max_segments((int)E, (int)A));
     w.x_sorted = take(A * H * 2);
     w.h = take(A * (size_t)c.inter * 2);
     w.h_shared = take((size_t)T * c.shared_inter * 2);

@@ -42,6 +42,7 @@
 // overlaps the routing kernels; everything produced inside the layer is touched after it.
 #include <cuda.h>
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "common.cuh"
@@ -63,8 +64,10 @@ struct FfnArgs {
     int K[2];      // reduction length per group kind
     __nv_bfloat16 *out[2];
     int out_ld[2];
-    const int32_t *plan_header;  // [0] = number of segments
+    const int32_t *plan_header;  // [0] = number of segments, [1] = number of segment pairs
     const Segment *seg;
+    const int32_t *pair_first;   // plan index of every pair's first segment
+    int round_robin;             // routed work dealt as (pair, tile) items instead of ranges
     int32_t *status;
     int T;             // token rows (the shared expert's group)
     int with_shared;   // shared expert present in this launch
@@ -279,14 +282,20 @@ struct ItemWalk {
     const int max_units;
     // shared expert: units (tile, segment pair) sj, sj + grid, ... of shared_tiles * pairs_s
     int sj, Us, s_base, s_rem, nseg_s, pairs_s;
-    // routed groups: from (fs, u) to (fs_hi, u_hi); fs = plan index of a group's first segment
+    // routed groups, range mode: from (fs, u) to (fs_hi, u_hi); fs = plan index of a group's
+    // first segment.  Round-robin mode: items ri, ri + grid, ... of n_pairs * ntiles, where
+    // item i is tile (i % ntiles) of pair (i / ntiles): the tiles of one pair run on
+    // neighbouring CTAs at the same time and share the pair's token rows in L2.
     int R0, nseg_total, fs, u, fs_hi, u_hi;
+    long long ri, r_items;
+    int ntiles;
     bool synced, group_loaded;
     // current group and tile
     Segment sg;
     int g_nseg, g_u_end;
     bool have_tile;
     int t_grp, t_expert, t_u0, t_h, t_row0, t_n, t_s, t_s_end;
+    bool t_once;  // the tile's weights are read by this pass over it only
 
     __device__ ItemWalk(const FfnArgs &args, bool already_synced)
         : a(args), max_units(args.max_tile >> 4), synced(false), group_loaded(false), have_tile(false)
@@ -299,6 +308,8 @@ struct ItemWalk {
         pairs_s = (nseg_s + 1) >> 1;
         R0 = a.rows[0] >> 4;
         nseg_total = fs = u = fs_hi = u_hi = 0;
+        ntiles = (R0 + max_units - 1) / max_units;
+        ri = r_items = 0;
         if (already_synced)
             sync(false);
     }
@@ -341,9 +352,17 @@ struct ItemWalk {
         if (wait)
             griddep_wait();
         nseg_total = a.plan_header[0];
-        const long long P = (long long)nseg_total * R0;
-        boundary(routed_bound(blockIdx.x, P), fs, u);
-        boundary(routed_bound(blockIdx.x + 1, P), fs_hi, u_hi);
+        if (a.round_robin) {
+            // continue the round-robin where the shared expert's units left off
+            const int G = gridDim.x;
+            const int n_shared = a.shared_tiles * pairs_s;
+            r_items = (long long)a.plan_header[1] * ntiles;
+            ri = ((int)blockIdx.x - n_shared % G + G) % G;
+        } else {
+            const long long P = (long long)nseg_total * R0;
+            boundary(routed_bound(blockIdx.x, P), fs, u);
+            boundary(routed_bound(blockIdx.x + 1, P), fs_hi, u_hi);
+        }
         synced = true;
     }
     // false when this CTA has no further item
@@ -360,7 +379,7 @@ struct ItemWalk {
                     it.n = min(FF_SEG, t_n - t_s * FF_SEG);
                     // segments 2q and 2q+1 of a tile form a pair
                     it.role = (t_s & 1) ? 2 : (t_s + 1 < t_s_end ? 1 : 0);
-                    it.w_once = t_grp == 0 ? (t_s_end <= 2) : (nseg_s <= 2);
+                    it.w_once = t_once;
                     ++t_s;
                     return true;
                 }
@@ -376,12 +395,33 @@ struct ItemWalk {
                 t_n = a.T;
                 t_s = 2 * q;
                 t_s_end = min(nseg_s, 2 * q + 2);
+                t_once = nseg_s <= 2;
                 sj += gridDim.x;
                 have_tile = true;
                 continue;
             }
             if (!synced)
                 sync(true);
+            if (a.round_robin) {
+                if (ri >= r_items)
+                    return false;
+                const int q = (int)(ri / ntiles), tile = (int)(ri - (long long)q * ntiles);
+                const int sidx = a.pair_first[q];
+                sg = a.seg[sidx];
+                g_nseg = (sg.n + FF_SEG - 1) / FF_SEG;
+                t_u0 = tile * max_units;
+                t_h = min(max_units, R0 - t_u0);
+                t_grp = 0;
+                t_expert = sg.expert;
+                t_row0 = sg.row0;
+                t_n = sg.n;
+                t_s = sidx - sg.first_seg;
+                t_s_end = min(g_nseg, t_s + 2);
+                t_once = g_nseg <= 2;
+                ri += gridDim.x;
+                have_tile = true;
+                continue;
+            }
             if (fs >= nseg_total || (fs == fs_hi && u >= u_hi))
                 return false;
             if (!group_loaded) {
@@ -399,6 +439,7 @@ struct ItemWalk {
                 t_n = sg.n;
                 t_s = 0;
                 t_s_end = g_nseg;
+                t_once = g_nseg <= 2;
                 u += t_h;
                 have_tile = true;
                 continue;
@@ -915,6 +956,28 @@ static void ffn_geometry(int T, FfnArgs &a)
     a.n_w_slots = ns;
 }
 
+// Range mode keeps every CTA alone on "its" groups, perfectly levelled.  It loses when
+//  - a range is shorter than a few tiles: its two ends are partial tiles, and a tile of any
+//    height costs K/16 tensor-core instructions, so short ranges turn issue-bound;
+//  - the token rows of `grid` groups do not fit in L2 beside the weight stream (large T): every
+//    tile would fetch its group's rows from HBM again.
+// Then, and when there are so many tiles per CTA that the last wave hardly matters, the routed
+// work is dealt round-robin as (pair, tile) items: full tiles only, and the CTAs work on a few
+// groups at a time.
+static bool use_round_robin(const moe_config_t &c, int T, int rows_routed, int K_routed, int max_tile,
+                            int grid)
+{
+    const char *force = getenv("MOE_FF_RR");
+    if (force)
+        return force[0] == '1';
+    const double n_act = expected_active_experts(c.n_experts, c.top_k, T);
+    const double rows_per_group = (double)T * c.top_k / n_act;
+    const double pairs = n_act * ceil(ceil(rows_per_group / FF_SEG) / 2.0);
+    const double tiles_per_cta = pairs * ((rows_routed + max_tile - 1) / max_tile) / grid;
+    const double token_bytes = rows_per_group * K_routed * 2.0 * grid;
+    return tiles_per_cta < 3.0 || tiles_per_cta >= 12.0 || token_bytes > 200.0 * 1024 * 1024;
+}
+
 template <bool GATED>
 static cudaError_t launch_ffn(FfnArgs &a, const FfnMaps &maps, cudaStream_t s)
 {
@@ -967,6 +1030,8 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
     a.out_ld[1] = c.shared_inter;
     a.plan_header = plan.header;
     a.seg = plan.seg;
+    a.pair_first = plan.pair_first;
+    a.round_robin = use_round_robin(c, T, c.inter, c.hidden, a.max_tile, ffn_grid()) ? 1 : 0;
     a.status = status;
     a.T = T;
     a.with_shared = with_shared ? 1 : 0;
@@ -1002,6 +1067,8 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
     a.out_ld[0] = a.out_ld[1] = c.hidden;
     a.plan_header = plan.header;
     a.seg = plan.seg;
+    a.pair_first = plan.pair_first;
+    a.round_robin = use_round_robin(c, T, c.hidden, c.inter, a.max_tile, ffn_grid()) ? 1 : 0;
     a.status = status;
     a.T = T;
     a.with_shared = with_shared ? 1 : 0;

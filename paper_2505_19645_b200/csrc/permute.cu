@@ -76,6 +76,18 @@ __device__ void build_plan(const int *cnt_sh, const int *off_sh, int *scan, int 
         plan.header[0] = *total;
         status[0] = 0;  // device status word: cleared at the start of every FFN pass
     }
+    // pairs: segments 2q and 2q+1 of a group
+    const int first = nseg > 0 ? scan[tid] : 0;
+    const int npair = (nseg + 1) >> 1;
+    __syncthreads();
+    if (tid < MOE_MAX_EXPERTS)
+        scan[tid] = npair;
+    __syncthreads();
+    block_exclusive_scan(scan, tmp, E, total);
+    for (int q = 0; q < npair; ++q)
+        plan.pair_first[scan[tid] + q] = first + 2 * q;
+    if (tid == 0)
+        plan.header[1] = *total;
 }
 
 // Every CTA rebuilds the (tiny) histogram and scan for itself, so no grid-wide
