@@ -10,7 +10,7 @@ constexpr int CB_THREADS = 256;
 __global__ void __launch_bounds__(CB_THREADS)
 combine_kernel(const __nv_bfloat16 *__restrict__ y, const int32_t *__restrict__ inv_perm,
                const float *__restrict__ topk_w, const __nv_bfloat16 *__restrict__ shared_y,
-               const float *__restrict__ shared_scale, int T, int H, int k,
+               int shared_parts, const float *__restrict__ shared_scale, int T, int H, int k,
                __nv_bfloat16 *__restrict__ out)
 {
     griddep_launch();
@@ -40,15 +40,18 @@ combine_kernel(const __nv_bfloat16 *__restrict__ y, const int32_t *__restrict__ 
         }
         if (shared_y) {
             const float s = shared_scale ? shared_scale[t] : 1.0f;
-            const uint4 v = *reinterpret_cast<const uint4 *>(shared_y + (size_t)t * H + h);
-            acc[0] = fmaf(s, bf16_lo(v.x), acc[0]);
-            acc[1] = fmaf(s, bf16_hi(v.x), acc[1]);
-            acc[2] = fmaf(s, bf16_lo(v.y), acc[2]);
-            acc[3] = fmaf(s, bf16_hi(v.y), acc[3]);
-            acc[4] = fmaf(s, bf16_lo(v.z), acc[4]);
-            acc[5] = fmaf(s, bf16_hi(v.z), acc[5]);
-            acc[6] = fmaf(s, bf16_lo(v.w), acc[6]);
-            acc[7] = fmaf(s, bf16_hi(v.w), acc[7]);
+            for (int part = 0; part < shared_parts; ++part) {
+                const uint4 v = *reinterpret_cast<const uint4 *>(
+                    shared_y + ((size_t)part * T + t) * H + h);
+                acc[0] = fmaf(s, bf16_lo(v.x), acc[0]);
+                acc[1] = fmaf(s, bf16_hi(v.x), acc[1]);
+                acc[2] = fmaf(s, bf16_lo(v.y), acc[2]);
+                acc[3] = fmaf(s, bf16_hi(v.y), acc[3]);
+                acc[4] = fmaf(s, bf16_lo(v.z), acc[4]);
+                acc[5] = fmaf(s, bf16_hi(v.z), acc[5]);
+                acc[6] = fmaf(s, bf16_lo(v.w), acc[6]);
+                acc[7] = fmaf(s, bf16_hi(v.w), acc[7]);
+            }
         }
         uint4 o;
         __nv_bfloat162 p;
@@ -65,7 +68,7 @@ combine_kernel(const __nv_bfloat16 *__restrict__ y, const int32_t *__restrict__ 
 }
 
 cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, const int32_t *inv_perm,
-                           const float *topk_w, const __nv_bfloat16 *shared_y,
+                           const float *topk_w, const __nv_bfloat16 *shared_y, int shared_parts,
                            const float *shared_scale, int T, __nv_bfloat16 *out, cudaStream_t s)
 {
     const size_t total = (size_t)T * (c.hidden >> 3);
@@ -74,7 +77,7 @@ cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, const 
     if (blocks > cap)
         blocks = cap;
     return launch_pdl(combine_kernel, dim3((unsigned)blocks), dim3(CB_THREADS), 0, s, y, inv_perm,
-                      topk_w, shared_y, shared_scale, T, c.hidden, c.top_k, out);
+                      topk_w, shared_y, shared_parts, shared_scale, T, c.hidden, c.top_k, out);
 }
 
 }  // namespace moe

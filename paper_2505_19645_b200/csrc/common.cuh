@@ -58,11 +58,15 @@ struct Workspace {
     size_t h;             // bf16 [A, I]      SwiGLU intermediate, sorted order
     size_t h_shared;      // bf16 [T, I_s]
     size_t y;             // bf16 [A, H]      expert outputs, sorted order
-    size_t y_shared;      // bf16 [T, H]
+    size_t y_shared;      // bf16 [shared_down_parts, T, H]: partial sums per k chunk
     size_t total;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// k chunks the shared expert's down projection is split into inside moe_verify_layer (each
+// chunk is a work unit of its own and writes a partial [T,H] plane that the combine step sums)
+int shared_down_parts(const moe_config_t &c);
 
 inline Workspace workspace_layout(const moe_config_t &c, int T)
 {
@@ -92,7 +96,7 @@ inline Workspace workspace_layout(const moe_config_t &c, int T)
     w.h = take(A * (size_t)c.inter * 2);
     w.h_shared = take((size_t)T * c.shared_inter * 2);
     w.y = take(A * H * 2);
-    w.y_shared = take((size_t)T * H * 2);
+    w.y_shared = take((size_t)T * H * 2 * shared_down_parts(c));
     w.total = off;
     return w;
 }
@@ -124,13 +128,14 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
                               cudaStream_t s);
 cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T, PlanView plan,
                             bool with_shared, const __nv_bfloat16 *h, const __nv_bfloat16 *h_shared,
-                            __nv_bfloat16 *y, __nv_bfloat16 *y_shared, int32_t *status,
-                            cudaStream_t s);
+                            __nv_bfloat16 *y, __nv_bfloat16 *y_shared, int shared_parts,
+                            int32_t *status, cudaStream_t s);
 // token rows in sorted order (the token operand of the routed gate/up tiles)
 cudaError_t launch_gather_rows(const moe_config_t &c, const __nv_bfloat16 *x, const int32_t *perm,
                                int T, __nv_bfloat16 *x_sorted, cudaStream_t s);
+// shared_y may hold `shared_parts` partial planes [T,H] (k chunks of the down pass), summed here
 cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, const int32_t *inv_perm,
-                           const float *topk_w, const __nv_bfloat16 *shared_y,
+                           const float *topk_w, const __nv_bfloat16 *shared_y, int shared_parts,
                            const float *shared_scale, int T, __nv_bfloat16 *out, cudaStream_t s);
 
 int sm_count();
@@ -147,7 +152,7 @@ PlanView plan_view(char *ws, const Workspace &L);
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
                      const int32_t *offsets, const int32_t *perm, __nv_bfloat16 *y,
                      __nv_bfloat16 *shared_y, char *ws, const Workspace &L, cudaStream_t s,
-                     int &launches, bool plan_ready = false);
+                     int &launches, bool plan_ready = false, int shared_parts = 1);
 
 // ---------------------------------------------------------------------------------------
 // Device helpers.

@@ -71,6 +71,11 @@ struct FfnArgs {
     int32_t *status;
     int T;             // token rows (the shared expert's group)
     int with_shared;   // shared expert present in this launch
+    int shared_ksplit;   // k chunks of the shared expert's reduction (down pass; 1 = whole K):
+                         // chunk s covers [s * shared_kchunk, ...) and writes its partial sums
+                         // to out[1] + s * shared_part_stride
+    int shared_kchunk;   // multiple of 128
+    long long shared_part_stride;  // elements
     int shared_tiles;  // tiles of the shared expert's rows; (tile, segment pair) units are dealt
                        // round-robin to the CTAs; the first (units % tiles) tiles have one
                        // 16-row unit more
@@ -271,6 +276,8 @@ struct Item {
     int n;       // token rows, 1..FF_SEG
     int role;    // 0 single, 1 first of a pair, 2 second of a pair (shares the first's tile)
     int w_once;  // the tile's weights are read by this item (or pair) only
+    int k0, k1;  // reduction range [k0, k1)
+    long long out_off;  // element offset of this item's output plane (k chunk) in out[grp]
 };
 
 // Walks the items of one CTA: its units of the shared expert first (they depend on nothing
@@ -281,7 +288,7 @@ struct ItemWalk {
     const FfnArgs &a;
     const int max_units;
     // shared expert: units (tile, segment pair) sj, sj + grid, ... of shared_tiles * pairs_s
-    int sj, Us, s_base, s_rem, nseg_s, pairs_s;
+    int sj, Us, s_base, s_rem, nseg_s, pairs_s, s_units;
     // routed groups, range mode: from (fs, u) to (fs_hi, u_hi); fs = plan index of a group's
     // first segment.  Round-robin mode: items ri, ri + grid, ... of n_pairs * ntiles, where
     // item i is tile (i % ntiles) of pair (i / ntiles): the tiles of one pair run on
@@ -296,6 +303,8 @@ struct ItemWalk {
     bool have_tile;
     int t_grp, t_expert, t_u0, t_h, t_row0, t_n, t_s, t_s_end;
     bool t_once;  // the tile's weights are read by this pass over it only
+    int t_k0, t_k1;
+    long long t_out_off;
 
     __device__ ItemWalk(const FfnArgs &args, bool already_synced)
         : a(args), max_units(args.max_tile >> 4), synced(false), group_loaded(false), have_tile(false)
@@ -306,6 +315,7 @@ struct ItemWalk {
         sj = blockIdx.x;
         nseg_s = (a.T + FF_SEG - 1) / FF_SEG;
         pairs_s = (nseg_s + 1) >> 1;
+        s_units = a.shared_tiles * a.shared_ksplit * pairs_s;
         R0 = a.rows[0] >> 4;
         nseg_total = fs = u = fs_hi = u_hi = 0;
         ntiles = (R0 + max_units - 1) / max_units;
@@ -321,11 +331,11 @@ struct ItemWalk {
     __device__ long long routed_bound(int c, long long P) const
     {
         const int G = gridDim.x;
-        const int r = (a.shared_tiles * pairs_s) % G;
+        const int r = s_units % G;
         if (r == 0)
             return P * c / G;
         const long long unit_cost =
-            (long long)(s_base + (s_rem ? 1 : 0)) * a.K[1] * nseg_s / pairs_s;
+            (long long)(s_base + (s_rem ? 1 : 0)) * (a.K[1] / a.shared_ksplit) * nseg_s / pairs_s;
         const long long p_cost = P * a.K[0];
         const int n_lo = G - r;
         if (p_cost <= unit_cost * n_lo)
@@ -355,7 +365,7 @@ struct ItemWalk {
         if (a.round_robin) {
             // continue the round-robin where the shared expert's units left off
             const int G = gridDim.x;
-            const int n_shared = a.shared_tiles * pairs_s;
+            const int n_shared = s_units;
             r_items = (long long)a.plan_header[1] * ntiles;
             ri = ((int)blockIdx.x - n_shared % G + G) % G;
         } else {
@@ -380,13 +390,20 @@ struct ItemWalk {
                     // segments 2q and 2q+1 of a tile form a pair
                     it.role = (t_s & 1) ? 2 : (t_s + 1 < t_s_end ? 1 : 0);
                     it.w_once = t_once;
+                    it.k0 = t_k0;
+                    it.k1 = t_k1;
+                    it.out_off = t_out_off;
                     ++t_s;
                     return true;
                 }
                 have_tile = false;
             }
-            if (sj < a.shared_tiles * pairs_s) {  // next unit of the shared expert
-                const int tile = sj / pairs_s, q = sj - tile * pairs_s;
+            if (sj < s_units) {  // next unit of the shared expert: (tile, k chunk, segment pair)
+                const int tc = sj / pairs_s, q = sj - tc * pairs_s;
+                const int tile = tc / a.shared_ksplit, chunk = tc - tile * a.shared_ksplit;
+                t_k0 = chunk * a.shared_kchunk;
+                t_k1 = min(a.K[1], t_k0 + a.shared_kchunk);
+                t_out_off = chunk * a.shared_part_stride;
                 t_u0 = tile * s_base + min(tile, s_rem);
                 t_h = s_base + (tile < s_rem ? 1 : 0);
                 t_grp = 1;
@@ -418,6 +435,9 @@ struct ItemWalk {
                 t_s = sidx - sg.first_seg;
                 t_s_end = min(g_nseg, t_s + 2);
                 t_once = g_nseg <= 2;
+                t_k0 = 0;
+                t_k1 = a.K[0];
+                t_out_off = 0;
                 ri += gridDim.x;
                 have_tile = true;
                 continue;
@@ -440,6 +460,9 @@ struct ItemWalk {
                 t_s = 0;
                 t_s_end = g_nseg;
                 t_once = g_nseg <= 2;
+                t_k0 = 0;
+                t_k1 = a.K[0];
+                t_out_off = 0;
                 u += t_h;
                 have_tile = true;
                 continue;
@@ -573,10 +596,10 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 }
                 if (it.role == 2)
                     continue;  // rides on the tile loaded for the first of its pair
-                const int K = args.K[it.grp];
+                const int K = it.k1;
                 const uint32_t tile_bytes = (uint32_t)it.h * 128u;
                 const int wrow = it.expert * args.rows[0] + it.f0;  // expert = 0 for the shared kind
-                for (int k0 = 0; k0 < K; k0 += 64 * kb) {
+                for (int k0 = it.k0; k0 < K; k0 += 64 * kb) {
                     const int nbox = min(kb, (K - k0 + 63) >> 6);
                     if (!mbar_wait(w_empty(slot), phase ^ 1u, abortp, args.status)) {
                         ok = false;
@@ -642,8 +665,8 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 if (nsub == 2 && !walk.next(it2))
                     break;  // cannot happen: a first is always followed by its second
                 const CUtensorMap *mx = &maps.x[it.grp];
-                const int K = args.K[it.grp];
-                for (int k0 = 0; ok && k0 < K; k0 += 64 * kb) {
+                const int K = it.k1;
+                for (int k0 = it.k0; ok && k0 < K; k0 += 64 * kb) {
                     const int nbox = min(kb, (K - k0 + 63) >> 6);
                     for (int sub = 0; sub < nsub; ++sub) {
                         const Item &cur = sub ? it2 : it;
@@ -716,8 +739,8 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 tc_fence_after();
                 const uint32_t tile_bytes = (uint32_t)it.h * 128u;
                 const uint32_t idesc = umma_idesc_bf16(NW * it.h);
-                const int K = args.K[it.grp];
-                for (int k0 = 0; ok && k0 < K; k0 += 64 * kb) {
+                const int K = it.k1;
+                for (int k0 = it.k0; ok && k0 < K; k0 += 64 * kb) {
                     const int nbox = min(kb, (K - k0 + 63) >> 6);
                     // the weight slot is multiplied with one or two segments' token entries
                     uint32_t xbase[2];
@@ -744,7 +767,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                         for (int b = 0; b < nbox; ++b) {
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
-                                const uint32_t accum = (k0 | b | q) != 0 ? 1u : 0u;
+                                const uint32_t accum = ((k0 - it.k0) | b | q) != 0 ? 1u : 0u;
                                 umma_bf16(d0,
                                           umma_desc_sw128(xbase[sub] + (uint32_t)(b * pieces[sub]) * FF_X_UNIT + q * 32),
                                           umma_desc_sw128(wbase + b * NW * tile_bytes + q * 32), idesc, accum);
@@ -792,7 +815,8 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             if (quarter * 32 < it.n) {
                 const int trow = quarter * 32 + lane;  // token row of this thread
                 const bool row_ok = trow < it.n;
-                __nv_bfloat16 *out = args.out[it.grp] + (size_t)(it.row0 + trow) * args.out_ld[it.grp] + it.f0;
+                __nv_bfloat16 *out =
+                    args.out[it.grp] + it.out_off + (size_t)(it.row0 + trow) * args.out_ld[it.grp] + it.f0;
                 const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * ACC_COLS);
                 for (int c = 0; c < it.h; c += 16) {
                     uint32_t g[16], u[16];
@@ -922,7 +946,8 @@ static int ffn_grid() { return sm_count(); }
 // instruction costs the same for any tile height, so tiles below 128 stacked rows (the N
 // operand) would make the pass issue-bound.
 static int shared_tile_count(const moe_config_t &c, int T, int rows_routed, int rows_shared,
-                             int K_routed, int K_shared, int min_tile, int max_tile, int grid)
+                             int K_routed, int K_shared, int ksplit, int min_tile, int max_tile,
+                             int grid)
 {
     const int nseg_s = (T + FF_SEG - 1) / FF_SEG;
     const int pairs_s = (nseg_s + 1) / 2;
@@ -931,7 +956,7 @@ static int shared_tile_count(const moe_config_t &c, int T, int rows_routed, int 
     const double n_act = expected_active_experts(c.n_experts, c.top_k, T);
     const double segs_r = n_act * ceil((double)T * c.top_k / n_act / FF_SEG);
     const double total = units * k_ratio * nseg_s + segs_r * (rows_routed >> 4);
-    int tu = (int)ceil(total / grid / (k_ratio * nseg_s / pairs_s));
+    int tu = (int)ceil(total / grid / (k_ratio / ksplit * nseg_s / pairs_s));
     if (tu < (min_tile >> 4))
         tu = min_tile >> 4;
     if (tu > (max_tile >> 4))
@@ -1009,8 +1034,10 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
     a.rows[1] = c.shared_inter;
     a.K[0] = a.K[1] = c.hidden;
     a.max_tile = 128;
+    a.shared_ksplit = 1;
+    a.shared_kchunk = (c.hidden + 127) / 128 * 128;
     a.shared_tiles = with_shared ? shared_tile_count(c, T, c.inter, c.shared_inter, c.hidden, c.hidden,
-                                                     64, 128, ffn_grid())
+                                                     1, 64, 128, ffn_grid())
                                  : 0;
     ffn_geometry(T, a);
     FfnMaps maps;
@@ -1038,10 +1065,18 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
     return launch_ffn<true>(a, maps, s);
 }
 
+int shared_down_parts(const moe_config_t &c)
+{
+    if (c.shared_inter < 2 * c.inter)
+        return 1;
+    const int s = c.shared_inter / c.inter;
+    return s > 8 ? 8 : s;
+}
+
 cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T, PlanView plan,
                             bool with_shared, const __nv_bfloat16 *h, const __nv_bfloat16 *h_shared,
-                            __nv_bfloat16 *y, __nv_bfloat16 *y_shared, int32_t *status,
-                            cudaStream_t s)
+                            __nv_bfloat16 *y, __nv_bfloat16 *y_shared, int shared_parts,
+                            int32_t *status, cudaStream_t s)
 {
     const uint64_t A = (uint64_t)T * c.top_k, H = c.hidden, E = c.n_experts;
     FfnArgs a{};
@@ -1049,8 +1084,12 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
     a.K[0] = c.inter;
     a.K[1] = c.shared_inter;
     a.max_tile = 256;
+    a.shared_ksplit = with_shared ? shared_parts : 1;
+    a.shared_kchunk = with_shared ? ((c.shared_inter + a.shared_ksplit - 1) / a.shared_ksplit + 127) / 128 * 128
+                                  : 128;
+    a.shared_part_stride = (long long)T * c.hidden;
     a.shared_tiles = with_shared ? shared_tile_count(c, T, c.hidden, c.hidden, c.inter, c.shared_inter,
-                                                     128, 256, ffn_grid())
+                                                     a.shared_ksplit, 128, 256, ffn_grid())
                                  : 0;
     ffn_geometry(T, a);
     FfnMaps maps;
