@@ -27,9 +27,10 @@ struct Segment {
 };
 
 // plan header (ints): [0] number of segments over all activated experts,
-//                     [1] number of segment pairs (segments 2q and 2q+1 of a group form a pair)
+//                     [1] number of segment pairs (segments 2q and 2q+1 of a group form a pair),
+//                     [2], [3] routed work claimed so far by the gate/up and the down pass
 struct PlanView {
-    int32_t *header;
+    int32_t *header;      // written by the plan; [2], [3] advanced by the FFN kernels
     Segment *seg;         // capacity max_segments()
     int32_t *pair_first;  // plan index of every pair's first segment, capacity max_segments()
 };

@@ -67,6 +67,7 @@ struct FfnArgs {
     const int32_t *plan_header;  // [0] = number of segments, [1] = number of segment pairs
     const Segment *seg;
     const int32_t *pair_first;   // plan index of every pair's first segment
+    int32_t *claim_counter;      // grid-wide: next unclaimed routed position / item of this pass
     int round_robin;             // routed work dealt as (pair, tile) items instead of ranges
     int32_t *status;
     int T;             // token rows (the shared expert's group)
@@ -280,23 +281,47 @@ struct Item {
     long long out_off;  // element offset of this item's output plane (k chunk) in out[grp]
 };
 
-// Walks the items of one CTA: its units of the shared expert first (they depend on nothing
-// the layer computes), then its range of the routed groups' rows.  The routed part needs the
-// segment plan, which the preceding kernels write: next() calls griddepcontrol.wait once
-// before it touches the plan (or before reporting the end).
+// Hand-over of the routed work a CTA claims at run time.  One thread of the CTA (the weight
+// producer) claims chunks from a grid-wide counter and publishes them in a small ring; the
+// other roles read the same sequence, so all roles walk identical items.
+constexpr int FF_CLAIMS = 4;      // ring entries
+constexpr int FF_CLAIM_READERS = 6;  // token producer, MMA issuer, 4 epilogue warps
+
+struct ClaimRing {
+    int *lo, *hi;              // shared memory [FF_CLAIMS]
+    uint32_t full0, empty0;    // shared addresses of the barrier arrays [FF_CLAIMS]
+    volatile int *abort_flag;
+    int32_t *status;
+};
+
+// Walks the items of one CTA: its units of the shared expert first (dealt round-robin: they
+// depend on nothing the layer computes), then chunks of the routed groups' work, claimed from
+// a grid-wide counter so that a CTA that is late or slow simply takes less.  The routed part
+// needs the segment plan, which the preceding kernels write: next() calls
+// griddepcontrol.wait once before it touches the plan (or before reporting the end).
+//
+// Routed work, range mode: positions (16 rows of one group for one of its segments, groups
+// laid end to end); a chunk is a run of positions whose ends are moved to tile boundaries, its
+// length shrinks as the work runs out (a third of the remaining per-CTA share, at least one
+// tile).  Round-robin mode: a chunk is one (segment pair, tile) item; consecutive items are
+// the tiles of one pair, which then run on many CTAs at once and share the pair's token rows
+// in L2.
 struct ItemWalk {
     const FfnArgs &a;
+    const ClaimRing &ring;
+    const bool claimer;    // this thread claims; all others follow the ring
+    const bool lead;       // this thread arrives on the ring's barriers for its role
+    const bool warp_wide;  // the role is run by all 32 lanes in lock step (epilogue warps)
     const int max_units;
-    // shared expert: units (tile, segment pair) sj, sj + grid, ... of shared_tiles * pairs_s
+    int n_claims;
+    // shared expert: units (tile, k chunk, segment pair) sj, sj + grid, ...
     int sj, Us, s_base, s_rem, nseg_s, pairs_s, s_units;
-    // routed groups, range mode: from (fs, u) to (fs_hi, u_hi); fs = plan index of a group's
-    // first segment.  Round-robin mode: items ri, ri + grid, ... of n_pairs * ntiles, where
-    // item i is tile (i % ntiles) of pair (i / ntiles): the tiles of one pair run on
-    // neighbouring CTAs at the same time and share the pair's token rows in L2.
+    // routed groups: current chunk from (fs, u) to (fs_hi, u_hi); fs = plan index of a
+    // group's first segment
     int R0, nseg_total, fs, u, fs_hi, u_hi;
-    long long ri, r_items;
+    long long P;
     int ntiles;
-    bool synced, group_loaded;
+    bool synced, group_loaded, have_chunk, finished;
     // current group and tile
     Segment sg;
     int g_nseg, g_u_end;
@@ -306,8 +331,12 @@ struct ItemWalk {
     int t_k0, t_k1;
     long long t_out_off;
 
-    __device__ ItemWalk(const FfnArgs &args, bool already_synced)
-        : a(args), max_units(args.max_tile >> 4), synced(false), group_loaded(false), have_tile(false)
+    __device__ ItemWalk(const FfnArgs &args, const ClaimRing &r, bool is_claimer, bool is_lead,
+                        bool is_warp_wide, bool already_synced)
+        : a(args), ring(r), claimer(is_claimer), lead(is_lead), warp_wide(is_warp_wide),
+          max_units(args.max_tile >> 4),
+          n_claims(0), synced(false), group_loaded(false), have_chunk(false), finished(false),
+          have_tile(false)
     {
         Us = a.with_shared ? a.rows[1] >> 4 : 0;
         s_base = a.shared_tiles ? Us / a.shared_tiles : 0;
@@ -319,35 +348,14 @@ struct ItemWalk {
         R0 = a.rows[0] >> 4;
         nseg_total = fs = u = fs_hi = u_hi = 0;
         ntiles = (R0 + max_units - 1) / max_units;
-        ri = r_items = 0;
+        P = 0;
         if (already_synced)
             sync(false);
     }
-    // First routed position of CTA c.  CTAs [0, r) hold one shared unit more than CTAs [r, G);
-    // the routed positions first fill the second class up to the first, the rest is spread
-    // over everybody.  Costs are counted in (16 rows x 1 k element x 1 segment): a routed
-    // position costs K[0], a shared unit (tile height) * K[1] * (segments per unit).  Integer
-    // arithmetic only, so every role of every CTA derives the same bounds.
-    __device__ long long routed_bound(int c, long long P) const
-    {
-        const int G = gridDim.x;
-        const int r = s_units % G;
-        if (r == 0)
-            return P * c / G;
-        const long long unit_cost =
-            (long long)(s_base + (s_rem ? 1 : 0)) * (a.K[1] / a.shared_ksplit) * nseg_s / pairs_s;
-        const long long p_cost = P * a.K[0];
-        const int n_lo = G - r;
-        if (p_cost <= unit_cost * n_lo)
-            return c < r ? 0 : P * (c - r) / n_lo;
-        const long long extra = p_cost - unit_cost * n_lo;  // spread over all G CTAs
-        return (extra * c + unit_cost * G * (c > r ? c - r : 0)) / ((long long)G * a.K[0]);
-    }
-    // position p (in units of 16 rows x one segment, groups laid end to end, each group's
-    // units repeated for all its segments) -> (group, row unit)
+    // position p -> (group, row unit rounded down to a tile boundary of the group)
     __device__ void boundary(long long p, int &fs_out, int &u_out) const
     {
-        if (p >= (long long)nseg_total * R0) {
+        if (p >= P) {
             fs_out = nseg_total;
             u_out = 0;
             return;
@@ -355,25 +363,50 @@ struct ItemWalk {
         const Segment s = a.seg[(int)(p / R0)];
         const int ns = (s.n + FF_SEG - 1) / FF_SEG;
         fs_out = s.first_seg;
-        u_out = (int)((p - (long long)s.first_seg * R0) / ns);
+        u_out = (int)((p - (long long)s.first_seg * R0) / ns) / max_units * max_units;
     }
     __device__ void sync(bool wait)
     {
         if (wait)
             griddep_wait();
         nseg_total = a.plan_header[0];
-        if (a.round_robin) {
-            // continue the round-robin where the shared expert's units left off
-            const int G = gridDim.x;
-            const int n_shared = s_units;
-            r_items = (long long)a.plan_header[1] * ntiles;
-            ri = ((int)blockIdx.x - n_shared % G + G) % G;
-        } else {
-            const long long P = (long long)nseg_total * R0;
-            boundary(routed_bound(blockIdx.x, P), fs, u);
-            boundary(routed_bound(blockIdx.x + 1, P), fs_hi, u_hi);
-        }
+        P = a.round_robin ? (long long)a.plan_header[1] * ntiles : (long long)nseg_total * R0;
         synced = true;
+    }
+    // Next chunk [lo, hi) of the routed work; false when none is left (or on abort).
+    __device__ bool acquire(int &lo, int &hi)
+    {
+        const int slot = n_claims % FF_CLAIMS;
+        const uint32_t par = (uint32_t)(n_claims / FF_CLAIMS) & 1u;
+        ++n_claims;
+        if (claimer) {
+            int size = 1;
+            if (!a.round_robin) {
+                const long long left = P - *reinterpret_cast<volatile int32_t *>(a.claim_counter);
+                const long long guided = left / (3 * (long long)gridDim.x);
+                size = (int)(guided > max_units ? guided : max_units);
+            }
+            lo = atomicAdd(a.claim_counter, size);
+            hi = (int)(lo + (long long)size < P ? lo + size : P);
+            if (lo >= P)
+                lo = hi = -1;
+            if (!mbar_wait(ring.empty0 + 8u * slot, par ^ 1u, ring.abort_flag, ring.status))
+                return false;
+            ring.lo[slot] = lo;
+            ring.hi[slot] = hi;
+            __threadfence_block();
+            mbar_arrive(ring.full0 + 8u * slot);
+        } else {
+            if (!mbar_wait(ring.full0 + 8u * slot, par, ring.abort_flag, ring.status))
+                return false;
+            lo = ring.lo[slot];
+            hi = ring.hi[slot];
+            if (warp_wide)
+                __syncwarp();  // every lane has read the entry before it is released
+            if (lead)
+                mbar_arrive(ring.empty0 + 8u * slot);
+        }
+        return lo >= 0;
     }
     // false when this CTA has no further item
     __device__ bool next(Item &it)
@@ -419,31 +452,44 @@ struct ItemWalk {
             }
             if (!synced)
                 sync(true);
-            if (a.round_robin) {
-                if (ri >= r_items)
+            if (finished)
+                return false;
+            if (!have_chunk) {
+                int lo, hi;
+                if (!acquire(lo, hi)) {
+                    finished = true;
                     return false;
-                const int q = (int)(ri / ntiles), tile = (int)(ri - (long long)q * ntiles);
-                const int sidx = a.pair_first[q];
-                sg = a.seg[sidx];
-                g_nseg = (sg.n + FF_SEG - 1) / FF_SEG;
-                t_u0 = tile * max_units;
-                t_h = min(max_units, R0 - t_u0);
-                t_grp = 0;
-                t_expert = sg.expert;
-                t_row0 = sg.row0;
-                t_n = sg.n;
-                t_s = sidx - sg.first_seg;
-                t_s_end = min(g_nseg, t_s + 2);
-                t_once = g_nseg <= 2;
-                t_k0 = 0;
-                t_k1 = a.K[0];
-                t_out_off = 0;
-                ri += gridDim.x;
-                have_tile = true;
+                }
+                if (a.round_robin) {
+                    // one (pair, tile) item
+                    const int q = lo / ntiles, tile = lo - q * ntiles;
+                    const int sidx = a.pair_first[q];
+                    sg = a.seg[sidx];
+                    g_nseg = (sg.n + FF_SEG - 1) / FF_SEG;
+                    t_u0 = tile * max_units;
+                    t_h = min(max_units, R0 - t_u0);
+                    t_grp = 0;
+                    t_expert = sg.expert;
+                    t_row0 = sg.row0;
+                    t_n = sg.n;
+                    t_s = sidx - sg.first_seg;
+                    t_s_end = min(g_nseg, t_s + 2);
+                    t_once = g_nseg <= 2;
+                    t_k0 = 0;
+                    t_k1 = a.K[0];
+                    t_out_off = 0;
+                    have_tile = true;
+                    continue;
+                }
+                boundary(lo, fs, u);
+                boundary(hi, fs_hi, u_hi);
+                group_loaded = false;
+                have_chunk = true;
+            }
+            if (fs >= nseg_total || fs > fs_hi || (fs == fs_hi && u >= u_hi)) {
+                have_chunk = false;  // chunk exhausted (or empty after rounding)
                 continue;
             }
-            if (fs >= nseg_total || (fs == fs_hi && u >= u_hi))
-                return false;
             if (!group_loaded) {
                 sg = a.seg[fs];
                 g_nseg = (sg.n + FF_SEG - 1) / FF_SEG;
@@ -524,9 +570,10 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
     constexpr int NW = GATED ? 2 : 1;  // weight matrices stacked in one N operand
 
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[2 * FF_MAX_W_SLOTS + 2 * FF_X_ENTRIES + 4];
+    __shared__ uint64_t bars[2 * FF_MAX_W_SLOTS + 2 * FF_X_ENTRIES + 4 + 2 * FF_CLAIMS];
     __shared__ uint32_t tmem_base_holder;
     __shared__ int abort_flag;
+    __shared__ int claim_lo[FF_CLAIMS], claim_hi[FF_CLAIMS];
 
     const int NS = args.n_w_slots;
     const int kb = args.kboxes;
@@ -541,6 +588,8 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
     auto x_empty = [&](int s) { return bar0 + 8u * (2 * FF_MAX_W_SLOTS + FF_X_ENTRIES + s); };
     auto acc_full = [&](int b) { return bar0 + 8u * (2 * FF_MAX_W_SLOTS + 2 * FF_X_ENTRIES + b); };
     auto acc_empty = [&](int b) { return bar0 + 8u * (2 * FF_MAX_W_SLOTS + 2 * FF_X_ENTRIES + 2 + b); };
+    const uint32_t claim_full0 = bar0 + 8u * (2 * FF_MAX_W_SLOTS + 2 * FF_X_ENTRIES + 4);
+    const uint32_t claim_empty0 = claim_full0 + 8u * FF_CLAIMS;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -558,6 +607,10 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             mbar_init(acc_full(b), 1);
             mbar_init(acc_empty(b), 4);
         }
+        for (int i = 0; i < FF_CLAIMS; ++i) {
+            mbar_init(claim_full0 + 8u * i, 1);
+            mbar_init(claim_empty0 + 8u * i, FF_CLAIM_READERS);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -573,6 +626,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_holder;
     volatile int *abortp = &abort_flag;
+    const ClaimRing claims{claim_lo, claim_hi, claim_full0, claim_empty0, abortp, args.status};
 
     if (warp == 0) {
         // ---------------- weight producer ----------------
@@ -580,7 +634,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             // gate/up pass: the shared expert's weights and x are the caller's inputs, so those
             // items run before the wait.  Down pass: every weight tile may be fetched ahead --
             // the launch order guarantees that the plan is complete when this kernel starts.
-            ItemWalk walk(args, !GATED);
+            ItemWalk walk(args, claims, true, false, false, !GATED);
             const uint64_t pol_once = l2_policy_evict_first();
             bool launched = !GATED;
             if (!GATED)
@@ -650,7 +704,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             // down pass: h is written by the preceding kernel
             if (!GATED)
                 griddep_wait();
-            ItemWalk walk(args, !GATED);
+            ItemWalk walk(args, claims, false, true, false, !GATED);
             XRingWalk ring(args.x_units);
             const uint64_t pol_keep = l2_policy_evict_last();
             int released = 0;          // entries known to have been consumed
@@ -714,7 +768,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            ItemWalk walk(args, !GATED);
+            ItemWalk walk(args, claims, false, true, false, !GATED);
             XRingWalk ring(args.x_units);
             int sw = 0;
             uint32_t pw = 0;
@@ -795,7 +849,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
         if (!GATED)
             griddep_wait();
         const int quarter = warp & 3;  // TMEM lanes 32*quarter .. +31 belong to this warp
-        ItemWalk walk(args, !GATED);
+        ItemWalk walk(args, claims, false, lane == 0, true, !GATED);
         int n_items = 0;
         Item it;
         for (;;) {
@@ -1058,6 +1112,7 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
     a.plan_header = plan.header;
     a.seg = plan.seg;
     a.pair_first = plan.pair_first;
+    a.claim_counter = plan.header + 2;
     a.round_robin = use_round_robin(c, T, c.inter, c.hidden, a.max_tile, ffn_grid()) ? 1 : 0;
     a.status = status;
     a.T = T;
@@ -1107,6 +1162,7 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
     a.plan_header = plan.header;
     a.seg = plan.seg;
     a.pair_first = plan.pair_first;
+    a.claim_counter = plan.header + 3;
     a.round_robin = use_round_robin(c, T, c.hidden, c.inter, a.max_tile, ffn_grid()) ? 1 : 0;
     a.status = status;
     a.T = T;

@@ -86,8 +86,11 @@ __device__ void build_plan(const int *cnt_sh, const int *off_sh, int *scan, int 
     block_exclusive_scan(scan, tmp, E, total);
     for (int q = 0; q < npair; ++q)
         plan.pair_first[scan[tid] + q] = first + 2 * q;
-    if (tid == 0)
+    if (tid == 0) {
         plan.header[1] = *total;
+        plan.header[2] = 0;  // work claimed so far by the gate/up pass ...
+        plan.header[3] = 0;  // ... and by the down pass
+    }
 }
 
 // Every CTA rebuilds the (tiny) histogram and scan for itself, so no grid-wide
