@@ -87,10 +87,10 @@ struct FfnArgs {
     int x_units;       // token ring size in FF_X_UNIT units
 };
 
-// Tensor maps of one pass: weights [kind][matrix][box height], token operand [kind].
+// Tensor maps of one pass: weights [kind][matrix][box height], token operand [kind][box height].
 struct FfnMaps {
     CUtensorMap w[2][2][FF_HEIGHTS];
-    CUtensorMap x[2];
+    CUtensorMap x[2][FF_HEIGHTS];
 };
 
 // ---- PTX wrappers ----------------------------------------------------------------------
@@ -718,7 +718,6 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 const int nsub = it.role == 1 ? 2 : 1;
                 if (nsub == 2 && !walk.next(it2))
                     break;  // cannot happen: a first is always followed by its second
-                const CUtensorMap *mx = &maps.x[it.grp];
                 const int K = it.k1;
                 for (int k0 = it.k0; ok && k0 < K; k0 += 64 * kb) {
                     const int nbox = min(kb, (K - k0 + 63) >> 6);
@@ -750,10 +749,20 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                         v_cur = v_end;
                         const uint32_t base = ring_x + (uint32_t)at * FF_X_UNIT;
                         mbar_expect_tx(x_full(e), (uint32_t)(nbox * pieces) * FF_X_UNIT);
-                        for (int b = 0; b < nbox; ++b)
-                            for (int p = 0; p < pieces; ++p)
-                                tma_load_2d_hint(base + (uint32_t)(b * pieces + p) * FF_X_UNIT, mx, x_full(e),
-                                                 k0 + 64 * b, cur.row0 + 16 * p, pol_keep);
+                        for (int b = 0; b < nbox; ++b) {
+                            // the entry's rows as boxes of 128, 64, 32 and 16 rows
+                            uint32_t dst = base + (uint32_t)(b * pieces) * FF_X_UNIT;
+                            int row = cur.row0, rem = pieces << 4;
+                            while (rem > 0) {
+                                const int hi = rem >= 128 ? 0 : (rem >= 64 ? 1 : (rem >= 32 ? 2 : 3));
+                                const int bh = 128 >> hi;
+                                tma_load_2d_hint(dst, &maps.x[it.grp][hi], x_full(e), k0 + 64 * b, row,
+                                                 pol_keep);
+                                dst += (uint32_t)bh * 128u;
+                                row += bh;
+                                rem -= bh;
+                            }
+                        }
                     }
                 }
             }
@@ -872,15 +881,29 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 __nv_bfloat16 *out =
                     args.out[it.grp] + it.out_off + (size_t)(it.row0 + trow) * args.out_ld[it.grp] + it.f0;
                 const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * ACC_COLS);
-                for (int c = 0; c < it.h; c += 16) {
-                    uint32_t g[16], u[16];
-                    tmem_ld16(t0 + c, g);
-                    if (GATED)
-                        tmem_ld16(t0 + it.h + c, u);
-                    tmem_ld_wait();
-                    if (row_ok) {
-                        epilogue_store8<GATED>(g, u, out + c);
-                        epilogue_store8<GATED>(g + 8, u + 8, out + c + 8);
+                // two register buffers: the TMEM load of the next 16 columns is in flight while
+                // the current 16 are converted and stored
+                uint32_t g[2][16], u[2][16];
+                tmem_ld16(t0, g[0]);
+                if (GATED)
+                    tmem_ld16(t0 + it.h, u[0]);
+#pragma unroll 1
+                for (int c = 0; c < it.h; c += 32) {
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        const int cc = c + 16 * half;
+                        if (cc < it.h) {
+                            tmem_ld_wait();
+                            if (cc + 16 < it.h) {
+                                tmem_ld16(t0 + cc + 16, g[half ^ 1]);
+                                if (GATED)
+                                    tmem_ld16(t0 + it.h + cc + 16, u[half ^ 1]);
+                            }
+                            if (row_ok) {
+                                epilogue_store8<GATED>(g[half], u[half], out + cc);
+                                epilogue_store8<GATED>(g[half] + 8, u[half] + 8, out + cc + 8);
+                            }
+                        }
                     }
                 }
             }
@@ -976,7 +999,7 @@ static bool make_map(CUtensorMap *m, const void *base, uint64_t rows, uint64_t c
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// the four box heights of one weight matrix
+// the four box heights of one matrix
 static bool make_weight_maps(CUtensorMap (&m)[FF_HEIGHTS], const void *base, uint64_t rows, uint64_t cols)
 {
     for (int i = 0; i < FF_HEIGHTS; ++i)
@@ -1024,9 +1047,12 @@ static int shared_tile_count(const moe_config_t &c, int T, int rows_routed, int 
 // three 128-row entries otherwise (a pair of segments needs two at once).
 static void ffn_geometry(int T, FfnArgs &a)
 {
-    a.kboxes = 2;
+    const char *ekb = getenv("MOE_FF_KBOXES"), *exr = getenv("MOE_FF_XRING_KB");
+    a.kboxes = ekb ? atoi(ekb) : 2;
     a.w_slot_bytes = 256 * 128 * a.kboxes;  // a full tile: 256 stacked rows per k box
-    const int x_ring_bytes = T > 64 ? 96 * 1024 : 32 * 1024;
+    int x_ring_bytes = T > 64 ? 96 * 1024 : 32 * 1024;
+    if (exr)
+        x_ring_bytes = atoi(exr) * 1024;
     a.x_units = x_ring_bytes / FF_X_UNIT;
     const int avail = FF_SMEM_LIMIT - 1024 - 512;  // alignment slack, static shared memory
     int ns = (avail - x_ring_bytes) / a.w_slot_bytes;
@@ -1098,11 +1124,11 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
     memset(&maps, 0, sizeof maps);
     bool ok = make_weight_maps(maps.w[0][0], w.w_gate, E * c.inter, H) &&
               make_weight_maps(maps.w[0][1], w.w_up, E * c.inter, H) &&
-              make_map(&maps.x[0], x_sorted, A, H, 16);
+              make_weight_maps(maps.x[0], x_sorted, A, H);
     if (with_shared)
         ok = ok && make_weight_maps(maps.w[1][0], w.ws_gate, c.shared_inter, H) &&
              make_weight_maps(maps.w[1][1], w.ws_up, c.shared_inter, H) &&
-             make_map(&maps.x[1], x, T, H, 16);
+             make_weight_maps(maps.x[1], x, T, H);
     if (!ok)
         return cudaErrorInvalidValue;
     a.out[0] = h;
@@ -1150,10 +1176,10 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
     FfnMaps maps;
     memset(&maps, 0, sizeof maps);
     bool ok = make_weight_maps(maps.w[0][0], w.w_down, E * H, c.inter) &&
-              make_map(&maps.x[0], h, A, c.inter, 16);
+              make_weight_maps(maps.x[0], h, A, c.inter);
     if (with_shared)
         ok = ok && make_weight_maps(maps.w[1][0], w.ws_down, H, c.shared_inter) &&
-             make_map(&maps.x[1], h_shared, T, c.shared_inter, 16);
+             make_weight_maps(maps.x[1], h_shared, T, c.shared_inter);
     if (!ok)
         return cudaErrorInvalidValue;
     a.out[0] = y;

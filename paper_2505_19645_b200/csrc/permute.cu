@@ -4,7 +4,7 @@
 
 namespace moe {
 
-constexpr int PERM_THREADS = 1024;  // 32 warps: one warp places one expert
+constexpr int PERM_THREADS = 1024;  // assignments per CTA, one per thread
 
 // Exclusive scan of vals[0..n) (n <= MOE_MAX_EXPERTS <= blockDim.x) in shared memory;
 // returns the total in *total.  All threads of the block must call it.  Warp shuffles inside
@@ -93,40 +93,87 @@ __device__ void build_plan(const int *cnt_sh, const int *off_sh, int *scan, int 
     }
 }
 
-// Every CTA rebuilds the (tiny) histogram and scan for itself, so no grid-wide
-// dependency is needed; CTA b then places experts 32b .. 32b+31, one warp each, walking
-// the assignments in ascending order (ballot + prefix popcount) -- stable by construction,
-// no atomics decide a position.  CTA 0 also writes counts / offsets / active / n_active and,
-// inside moe_verify_layer, the FFN segment plan (one launch fewer).
+// Adds one to hist[e] for every lane with a valid e.  With few experts a plain per-lane
+// atomic would serialise the block on a handful of counters, so the lanes of a warp that hold
+// the same expert are combined first (one atomic per distinct expert); with many experts the
+// match itself (one round per distinct value) costs more than the rare conflict.
+// All lanes of the warp must call it; `few` is uniform.
+__device__ __forceinline__ void warp_histogram_add(int *hist, int e, bool valid, bool few)
+{
+    if (few) {
+        const uint32_t peers = __match_any_sync(0xffffffffu, valid ? e : -1);
+        if (valid && (threadIdx.x & 31) == __ffs(peers) - 1)
+            atomicAdd(&hist[e], __popc(peers));
+    } else if (valid) {
+        atomicAdd(&hist[e], 1);  // a count does not depend on the order of the adds
+    }
+}
+
+// Stable counting sort of the assignments by expert.  CTA b owns assignments
+// [b * 1024, b * 1024 + 1024), one per thread.  Every CTA rebuilds the (small) histograms it
+// needs for itself -- all assignments for the expert offsets, those before its own chunk for
+// its starting ranks -- so no grid-wide dependency is needed.  Inside the chunk an
+// assignment's rank among those of its expert is (earlier warps' counts, from a per-warp
+// table) + (earlier lanes of its warp, from a match mask): ascending assignment id within
+// every expert by construction, no atomics decide a position.  CTA 0 also writes counts /
+// offsets / active / n_active and, inside moe_verify_layer, the FFN segment plan.
 __global__ void __launch_bounds__(PERM_THREADS)
 permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__restrict__ counts,
                int32_t *__restrict__ offsets, int32_t *__restrict__ perm,
                int32_t *__restrict__ inv_perm, int32_t *__restrict__ active,
                int32_t *__restrict__ n_active, int32_t *__restrict__ status, PlanView plan)
 {
-    __shared__ int hist[MOE_MAX_EXPERTS];
+    __shared__ int hist[MOE_MAX_EXPERTS];    // all assignments
+    __shared__ int before[MOE_MAX_EXPERTS];  // assignments of earlier chunks
     __shared__ int offs[MOE_MAX_EXPERTS];
-    __shared__ int flag[MOE_MAX_EXPERTS];
     __shared__ int tmp[MOE_MAX_EXPERTS];
+    __shared__ uint16_t wcount[PERM_THREADS / 32][MOE_MAX_EXPERTS];  // per warp of this chunk
     __shared__ int total;
     griddep_launch();
-    const int tid = threadIdx.x;
-    if (tid < MOE_MAX_EXPERTS)
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int chunk0 = blockIdx.x * PERM_THREADS;
+    if (tid < MOE_MAX_EXPERTS) {
         hist[tid] = 0;
+        before[tid] = 0;
+    }
+    for (int i = tid; i < (PERM_THREADS / 32) * MOE_MAX_EXPERTS / 2; i += PERM_THREADS)
+        reinterpret_cast<uint32_t *>(&wcount[0][0])[i] = 0u;
     griddep_wait();  // the expert indices come from the preceding kernel
     __syncthreads();
-    for (int a = tid; a < A; a += PERM_THREADS) {
-        const int e = topk_idx[a];
-        if (e >= 0 && e < E)
-            atomicAdd(&hist[e], 1);  // a count does not depend on the order of the adds
+    const bool few = E <= 32;
+    for (int a0 = 0; a0 < A; a0 += PERM_THREADS) {
+        const int a = a0 + tid;
+        const int e = a < A ? topk_idx[a] : -1;
+        const bool valid = e >= 0 && e < E;
+        warp_histogram_add(hist, e, valid, few);
+        if (a0 < chunk0)
+            warp_histogram_add(before, e, valid, few);
     }
+    // this thread's assignment: rank inside its warp, and its warp's counts
+    const int my_a = chunk0 + tid;
+    const int my_e = my_a < A ? topk_idx[my_a] : -1;
+    const bool my_valid = my_e >= 0 && my_e < E;
+    const uint32_t peers = __match_any_sync(0xffffffffu, my_valid ? my_e : -1);
+    const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+    if (my_valid && lane == __ffs(peers) - 1)
+        wcount[warp][my_e] = (uint16_t)__popc(peers);
     __syncthreads();
     if (tid < MOE_MAX_EXPERTS)
         offs[tid] = tid < E ? hist[tid] : 0;
     __syncthreads();
     block_exclusive_scan(offs, tmp, E, &total);
 
+    if (my_valid) {
+        int pos = offs[my_e] + before[my_e] + rank_in_warp;
+        for (int w = 0; w < warp; ++w)
+            pos += wcount[w][my_e];
+        perm[pos] = my_a;
+        inv_perm[my_a] = pos;
+    }
+
     if (blockIdx.x == 0) {
+        int *flag = before;  // CTA 0 has no earlier chunk: its table is free (all zero) now
+        __syncthreads();
         if (tid < E) {
             counts[tid] = hist[tid];
             offsets[tid] = offs[tid];
@@ -136,7 +183,7 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
         if (tid < MOE_MAX_EXPERTS)
             flag[tid] = (tid < E && hist[tid] > 0) ? 1 : 0;
         __syncthreads();
-        int my_flag = tid < E ? flag[tid] : 0;
+        const int my_flag = tid < E ? flag[tid] : 0;
         block_exclusive_scan(flag, tmp, E, &total);
         if (tid < E && my_flag)
             active[flag[tid]] = tid;
@@ -147,45 +194,18 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
         if (plan.header != nullptr)
             build_plan(hist, offs, flag, tmp, &total, E, status, plan);
     }
-
-    const int warp = tid >> 5, lane = tid & 31;
-    const int e = blockIdx.x * 32 + warp;
-    if (e >= E || hist[e] == 0)
-        return;
-    int base = offs[e];
-    const uint32_t lt_mask = (1u << lane) - 1u;
-    for (int a0 = 0; a0 < A; a0 += 128) {
-        int ev[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int a = a0 + u * 32 + lane;
-            ev[u] = a < A ? topk_idx[a] : -1;
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int a = a0 + u * 32 + lane;
-            const bool hit = ev[u] == e;
-            const uint32_t m = __ballot_sync(0xffffffffu, hit);
-            if (hit) {
-                const int pos = base + __popc(m & lt_mask);
-                perm[pos] = a;
-                inv_perm[a] = pos;
-            }
-            base += __popc(m);
-        }
-    }
 }
 
 cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int32_t *counts,
                            int32_t *offsets, int32_t *perm, int32_t *inv_perm, int32_t *active,
                            int32_t *n_active, cudaStream_t s, const PlanView *plan, int32_t *status)
 {
-    const int E = c.n_experts;
-    const int blocks = (E + 31) / 32;
+    const int A = T * c.top_k;
+    const int blocks = (A + PERM_THREADS - 1) / PERM_THREADS;
     PlanView pv{};
     if (plan)
         pv = *plan;
-    return launch_pdl(permute_kernel, dim3(blocks), dim3(PERM_THREADS), 0, s, idx, T * c.top_k, E,
+    return launch_pdl(permute_kernel, dim3(blocks), dim3(PERM_THREADS), 0, s, idx, A, c.n_experts,
                       counts, offsets, perm, inv_perm, active, n_active, status, pv);
 }
 

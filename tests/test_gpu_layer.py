@@ -37,6 +37,23 @@ def test_layer_parity_small_shapes(name, H, E, k, I, Is, score, renorm, sgate, B
     check_layer_against_oracle(shape, w, x, B, gamma)
 
 
+@pytest.mark.parametrize("mode", ["0", "1"])
+@pytest.mark.parametrize("name,H,E,k,I,Is,B,gamma", [
+    ("rr-shared", 512, 60, 4, 352, 1408, 13, 4),     # shared expert with a k-split down pass
+    ("rr-segments", 256, 4, 2, 384, 256, 100, 3),    # 200 rows per expert: segment pairs, 4 shared segments
+    ("rr-ragged", 160, 6, 3, 224, 96, 11, 6),        # tiles shorter than a box, k tails
+])
+def test_layer_parity_in_both_scheduling_modes(monkeypatch, mode, name, H, E, k, I, Is, B, gamma):
+    """The FFN kernels hand out the routed work either as chunks of consecutive tiles or as
+    single (segment pair, tile) items; MOE_FF_RR forces one of the two."""
+    monkeypatch.setenv("MOE_FF_RR", mode)
+    shape = wl.small_shape(name, H, E, k, I, Is, 0, 0, 1)
+    w = wl.make_weights(shape, 300 + E, "cuda")
+    T = B * (gamma + 1)
+    x = wl.make_tokens(shape, T, 400 + T, "cuda")
+    check_layer_against_oracle(shape, w, x, B, gamma)
+
+
 def test_layer_depends_on_token_count_only_and_is_deterministic():
     """layer(B, gamma) == layer(B*(gamma+1), 0) bit for bit; two runs and a run on another
     stream give identical routing, grouping and outputs."""
