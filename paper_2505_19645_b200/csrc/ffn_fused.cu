@@ -287,8 +287,9 @@ struct Item {
 constexpr int FF_CLAIMS = 4;      // ring entries
 constexpr int FF_CLAIM_READERS = 6;  // token producer, MMA issuer, 4 epilogue warps
 
+constexpr int FF_CLAIM_WORDS = 8;  // lo, hi, and (round-robin mode) the item's group, decoded
 struct ClaimRing {
-    int *lo, *hi;              // shared memory [FF_CLAIMS]
+    int *data;                 // shared memory [FF_CLAIMS][FF_CLAIM_WORDS]
     uint32_t full0, empty0;    // shared addresses of the barrier arrays [FF_CLAIMS]
     volatile int *abort_flag;
     int32_t *status;
@@ -321,7 +322,8 @@ struct ItemWalk {
     int R0, nseg_total, fs, u, fs_hi, u_hi;
     long long P;
     int ntiles;
-    bool synced, group_loaded, have_chunk, finished;
+    bool synced, group_loaded, have_chunk, finished, primed;
+    int next_lo, next_hi;  // claimer: the claim in flight
     // current group and tile
     Segment sg;
     int g_nseg, g_u_end;
@@ -336,6 +338,7 @@ struct ItemWalk {
         : a(args), ring(r), claimer(is_claimer), lead(is_lead), warp_wide(is_warp_wide),
           max_units(args.max_tile >> 4),
           n_claims(0), synced(false), group_loaded(false), have_chunk(false), finished(false),
+          primed(false), next_lo(-1), next_hi(-1),
           have_tile(false)
     {
         Us = a.with_shared ? a.rows[1] >> 4 : 0;
@@ -373,34 +376,70 @@ struct ItemWalk {
         P = a.round_robin ? (long long)a.plan_header[1] * ntiles : (long long)nseg_total * R0;
         synced = true;
     }
-    // Next chunk [lo, hi) of the routed work; false when none is left (or on abort).
-    __device__ bool acquire(int &lo, int &hi)
+    // Claims the next chunk from the grid-wide counter (claimer only).
+    __device__ void claim(int &lo, int &hi)
+    {
+        int size = 1;
+        if (!a.round_robin) {
+            const long long left = P - *reinterpret_cast<volatile int32_t *>(a.claim_counter);
+            const long long guided = left / (3 * (long long)gridDim.x);
+            size = (int)(guided > max_units ? guided : max_units);
+        }
+        lo = atomicAdd(a.claim_counter, size);
+        hi = (int)(lo + (long long)size < P ? lo + size : P);
+        if (lo >= P)
+            lo = hi = -1;
+    }
+    // Next chunk [lo, hi) of the routed work; false when none is left (or on abort).  In
+    // round-robin mode the chunk is one item and `grp` receives its group (the claimer looks
+    // it up once; the other roles take it from the ring instead of going to global memory).
+    // While plenty of work is left the claimer keeps one claim in flight beyond the one it
+    // hands out, so that the atomic's latency is not on the path of the weight stream.
+    __device__ bool acquire(int &lo, int &hi, Segment &grp, int &sidx)
     {
         const int slot = n_claims % FF_CLAIMS;
         const uint32_t par = (uint32_t)(n_claims / FF_CLAIMS) & 1u;
         ++n_claims;
+        int *e = ring.data + slot * FF_CLAIM_WORDS;
         if (claimer) {
-            int size = 1;
-            if (!a.round_robin) {
-                const long long left = P - *reinterpret_cast<volatile int32_t *>(a.claim_counter);
-                const long long guided = left / (3 * (long long)gridDim.x);
-                size = (int)(guided > max_units ? guided : max_units);
+            if (primed) {
+                lo = next_lo;
+                hi = next_hi;
+            } else {
+                claim(lo, hi);
             }
-            lo = atomicAdd(a.claim_counter, size);
-            hi = (int)(lo + (long long)size < P ? lo + size : P);
-            if (lo >= P)
-                lo = hi = -1;
+            // while plenty of work is left, the following claim is made now and consumed at
+            // the next call (near the end a claim held in reserve would starve another CTA)
+            primed = lo >= 0 &&
+                     P - *reinterpret_cast<volatile int32_t *>(a.claim_counter) > 4 * (long long)gridDim.x * (a.round_robin ? 1 : max_units);
+            if (primed)
+                claim(next_lo, next_hi);
+            sidx = 0;
+            if (lo >= 0 && a.round_robin) {
+                sidx = a.pair_first[lo / ntiles];
+                grp = a.seg[sidx];
+            }
             if (!mbar_wait(ring.empty0 + 8u * slot, par ^ 1u, ring.abort_flag, ring.status))
                 return false;
-            ring.lo[slot] = lo;
-            ring.hi[slot] = hi;
+            e[0] = lo;
+            e[1] = hi;
+            e[2] = sidx;
+            e[3] = grp.expert;
+            e[4] = grp.row0;
+            e[5] = grp.n;
+            e[6] = grp.first_seg;
             __threadfence_block();
             mbar_arrive(ring.full0 + 8u * slot);
         } else {
             if (!mbar_wait(ring.full0 + 8u * slot, par, ring.abort_flag, ring.status))
                 return false;
-            lo = ring.lo[slot];
-            hi = ring.hi[slot];
+            lo = e[0];
+            hi = e[1];
+            sidx = e[2];
+            grp.expert = e[3];
+            grp.row0 = e[4];
+            grp.n = e[5];
+            grp.first_seg = e[6];
             if (warp_wide)
                 __syncwarp();  // every lane has read the entry before it is released
             if (lead)
@@ -455,16 +494,14 @@ struct ItemWalk {
             if (finished)
                 return false;
             if (!have_chunk) {
-                int lo, hi;
-                if (!acquire(lo, hi)) {
+                int lo, hi, sidx;
+                if (!acquire(lo, hi, sg, sidx)) {
                     finished = true;
                     return false;
                 }
                 if (a.round_robin) {
                     // one (pair, tile) item
-                    const int q = lo / ntiles, tile = lo - q * ntiles;
-                    const int sidx = a.pair_first[q];
-                    sg = a.seg[sidx];
+                    const int tile = lo % ntiles;
                     g_nseg = (sg.n + FF_SEG - 1) / FF_SEG;
                     t_u0 = tile * max_units;
                     t_h = min(max_units, R0 - t_u0);
@@ -573,7 +610,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
     __shared__ uint64_t bars[2 * FF_MAX_W_SLOTS + 2 * FF_X_ENTRIES + 4 + 2 * FF_CLAIMS];
     __shared__ uint32_t tmem_base_holder;
     __shared__ int abort_flag;
-    __shared__ int claim_lo[FF_CLAIMS], claim_hi[FF_CLAIMS];
+    __shared__ int claim_data[FF_CLAIMS * FF_CLAIM_WORDS];
 
     const int NS = args.n_w_slots;
     const int kb = args.kboxes;
@@ -626,7 +663,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_holder;
     volatile int *abortp = &abort_flag;
-    const ClaimRing claims{claim_lo, claim_hi, claim_full0, claim_empty0, abortp, args.status};
+    const ClaimRing claims{claim_data, claim_full0, claim_empty0, abortp, args.status};
 
     if (warp == 0) {
         // ---------------- weight producer ----------------
@@ -789,17 +826,17 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 const int nsub = it.role == 1 ? 2 : 1;
                 if (nsub == 2 && !walk.next(it2))
                     break;  // cannot happen: a first is always followed by its second
+                // accumulator buffers: each is waited for right before its first instruction, so
+                // that the first segment of a pair starts while the epilogue still drains the
+                // other buffer
                 int buf[2];
-                for (int sub = 0; ok && sub < nsub; ++sub) {
+                uint32_t acc_par[2];
+                bool acc_ready[2] = {false, false};
+                for (int sub = 0; sub < nsub; ++sub) {
                     buf[sub] = n_items & 1;
-                    const uint32_t acc_phase = (uint32_t)(n_items >> 1) & 1u;
+                    acc_par[sub] = ((uint32_t)(n_items >> 1) & 1u) ^ 1u;
                     ++n_items;
-                    if (!mbar_wait(acc_empty(buf[sub]), acc_phase ^ 1u, abortp, args.status))
-                        ok = false;
                 }
-                if (!ok)
-                    break;
-                tc_fence_after();
                 const uint32_t tile_bytes = (uint32_t)it.h * 128u;
                 const uint32_t idesc = umma_idesc_bf16(NW * it.h);
                 const int K = it.k1;
@@ -826,6 +863,14 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                     tc_fence_after();
                     const uint32_t wbase = ring_w + sw * args.w_slot_bytes;
                     for (int sub = 0; sub < nsub; ++sub) {
+                        if (!acc_ready[sub]) {
+                            if (!mbar_wait(acc_empty(buf[sub]), acc_par[sub], abortp, args.status)) {
+                                ok = false;
+                                break;
+                            }
+                            tc_fence_after();
+                            acc_ready[sub] = true;
+                        }
                         const uint32_t d0 = tmem_base + (uint32_t)(buf[sub] * ACC_COLS);
                         for (int b = 0; b < nbox; ++b) {
 #pragma unroll
@@ -838,6 +883,8 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                         }
                         umma_commit(x_empty(xe[sub]));
                     }
+                    if (!ok)
+                        break;
                     umma_commit(w_empty(sw));  // reusable once these MMAs have read it
                     if (++sw == NS) {
                         sw = 0;
