@@ -21,36 +21,51 @@ combine_kernel(const __nv_bfloat16 *__restrict__ y, const int32_t *__restrict__ 
          i += (size_t)gridDim.x * CB_THREADS) {
         const int t = (int)(i / vec_per_row);
         const int h = (int)(i - (size_t)t * vec_per_row) << 3;
+        // the k rows of this token: positions and weights first, then all row pieces, so that
+        // the loads of one level are in flight together
+        int rows[MOE_MAX_TOPK];
+        float wts[MOE_MAX_TOPK];
+#pragma unroll
+        for (int j = 0; j < MOE_MAX_TOPK; ++j) {
+            rows[j] = j < k ? inv_perm[(size_t)t * k + j] : 0;
+            wts[j] = j < k ? topk_w[(size_t)t * k + j] : 0.f;
+        }
+        const float s = shared_y && shared_scale ? shared_scale[t] : 1.0f;
+        uint4 v[MOE_MAX_TOPK];
+#pragma unroll
+        for (int j = 0; j < MOE_MAX_TOPK; ++j)
+            if (j < k)
+                v[j] = *reinterpret_cast<const uint4 *>(y + (size_t)rows[j] * H + h);
         float acc[8];
 #pragma unroll
         for (int q = 0; q < 8; ++q)
             acc[q] = 0.f;
-        for (int j = 0; j < k; ++j) {
-            const int row = inv_perm[(size_t)t * k + j];
-            const float w = topk_w[(size_t)t * k + j];
-            const uint4 v = *reinterpret_cast<const uint4 *>(y + (size_t)row * H + h);
-            acc[0] = fmaf(w, bf16_lo(v.x), acc[0]);
-            acc[1] = fmaf(w, bf16_hi(v.x), acc[1]);
-            acc[2] = fmaf(w, bf16_lo(v.y), acc[2]);
-            acc[3] = fmaf(w, bf16_hi(v.y), acc[3]);
-            acc[4] = fmaf(w, bf16_lo(v.z), acc[4]);
-            acc[5] = fmaf(w, bf16_hi(v.z), acc[5]);
-            acc[6] = fmaf(w, bf16_lo(v.w), acc[6]);
-            acc[7] = fmaf(w, bf16_hi(v.w), acc[7]);
+#pragma unroll
+        for (int j = 0; j < MOE_MAX_TOPK; ++j) {
+            if (j < k) {
+                const float w = wts[j];
+                acc[0] = fmaf(w, bf16_lo(v[j].x), acc[0]);
+                acc[1] = fmaf(w, bf16_hi(v[j].x), acc[1]);
+                acc[2] = fmaf(w, bf16_lo(v[j].y), acc[2]);
+                acc[3] = fmaf(w, bf16_hi(v[j].y), acc[3]);
+                acc[4] = fmaf(w, bf16_lo(v[j].z), acc[4]);
+                acc[5] = fmaf(w, bf16_hi(v[j].z), acc[5]);
+                acc[6] = fmaf(w, bf16_lo(v[j].w), acc[6]);
+                acc[7] = fmaf(w, bf16_hi(v[j].w), acc[7]);
+            }
         }
         if (shared_y) {
-            const float s = shared_scale ? shared_scale[t] : 1.0f;
             for (int part = 0; part < shared_parts; ++part) {
-                const uint4 v = *reinterpret_cast<const uint4 *>(
+                const uint4 sv = *reinterpret_cast<const uint4 *>(
                     shared_y + ((size_t)part * T + t) * H + h);
-                acc[0] = fmaf(s, bf16_lo(v.x), acc[0]);
-                acc[1] = fmaf(s, bf16_hi(v.x), acc[1]);
-                acc[2] = fmaf(s, bf16_lo(v.y), acc[2]);
-                acc[3] = fmaf(s, bf16_hi(v.y), acc[3]);
-                acc[4] = fmaf(s, bf16_lo(v.z), acc[4]);
-                acc[5] = fmaf(s, bf16_hi(v.z), acc[5]);
-                acc[6] = fmaf(s, bf16_lo(v.w), acc[6]);
-                acc[7] = fmaf(s, bf16_hi(v.w), acc[7]);
+                acc[0] = fmaf(s, bf16_lo(sv.x), acc[0]);
+                acc[1] = fmaf(s, bf16_hi(sv.x), acc[1]);
+                acc[2] = fmaf(s, bf16_lo(sv.y), acc[2]);
+                acc[3] = fmaf(s, bf16_hi(sv.y), acc[3]);
+                acc[4] = fmaf(s, bf16_lo(sv.z), acc[4]);
+                acc[5] = fmaf(s, bf16_hi(sv.z), acc[5]);
+                acc[6] = fmaf(s, bf16_lo(sv.w), acc[6]);
+                acc[7] = fmaf(s, bf16_hi(sv.w), acc[7]);
             }
         }
         uint4 o;
