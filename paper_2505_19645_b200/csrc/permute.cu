@@ -115,8 +115,9 @@ __device__ __forceinline__ void warp_histogram_add(int *hist, int e, bool valid,
 // its starting ranks -- so no grid-wide dependency is needed.  Inside the chunk an
 // assignment's rank among those of its expert is (earlier warps' counts, from a per-warp
 // table) + (earlier lanes of its warp, from a match mask): ascending assignment id within
-// every expert by construction, no atomics decide a position.  CTA 0 also writes counts /
-// offsets / active / n_active and, inside moe_verify_layer, the FFN segment plan.
+// every expert by construction, no atomics decide a position.  One more CTA, which owns no
+// chunk, writes counts / offsets / active / n_active and, inside moe_verify_layer, the FFN
+// segment plan at the same time.
 __global__ void __launch_bounds__(PERM_THREADS)
 permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__restrict__ counts,
                int32_t *__restrict__ offsets, int32_t *__restrict__ perm,
@@ -131,7 +132,9 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
     __shared__ int total;
     griddep_launch();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int chunk0 = blockIdx.x * PERM_THREADS;
+    // the last CTA owns no chunk: it writes the tables and the plan while the others place
+    const bool tables_cta = blockIdx.x == gridDim.x - 1;
+    const int chunk0 = tables_cta ? 0 : blockIdx.x * PERM_THREADS;
     if (tid < MOE_MAX_EXPERTS) {
         hist[tid] = 0;
         before[tid] = 0;
@@ -151,7 +154,7 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
     }
     // this thread's assignment: rank inside its warp, and its warp's counts
     const int my_a = chunk0 + tid;
-    const int my_e = my_a < A ? topk_idx[my_a] : -1;
+    const int my_e = !tables_cta && my_a < A ? topk_idx[my_a] : -1;
     const bool my_valid = my_e >= 0 && my_e < E;
     const uint32_t peers = __match_any_sync(0xffffffffu, my_valid ? my_e : -1);
     const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
@@ -171,8 +174,8 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
         inv_perm[my_a] = pos;
     }
 
-    if (blockIdx.x == 0) {
-        int *flag = before;  // CTA 0 has no earlier chunk: its table is free (all zero) now
+    if (tables_cta) {
+        int *flag = before;  // this CTA counted no earlier chunk: the table is free (all zero)
         __syncthreads();
         if (tid < E) {
             counts[tid] = hist[tid];
@@ -201,7 +204,7 @@ cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int
                            int32_t *n_active, cudaStream_t s, const PlanView *plan, int32_t *status)
 {
     const int A = T * c.top_k;
-    const int blocks = (A + PERM_THREADS - 1) / PERM_THREADS;
+    const int blocks = (A + PERM_THREADS - 1) / PERM_THREADS + 1;  // + the tables CTA
     PlanView pv{};
     if (plan)
         pv = *plan;
