@@ -322,8 +322,8 @@ struct ItemWalk {
     int R0, nseg_total, fs, u, fs_hi, u_hi;
     long long P;
     int ntiles;
-    bool synced, group_loaded, have_chunk, finished, primed;
-    int next_lo, next_hi;  // claimer: the claim in flight
+    bool synced, group_loaded, have_chunk, finished, end_published;
+    int n_pub;  // claimer: chunks published so far
     // current group and tile
     Segment sg;
     int g_nseg, g_u_end;
@@ -338,7 +338,7 @@ struct ItemWalk {
         : a(args), ring(r), claimer(is_claimer), lead(is_lead), warp_wide(is_warp_wide),
           max_units(args.max_tile >> 4),
           n_claims(0), synced(false), group_loaded(false), have_chunk(false), finished(false),
-          primed(false), next_lo(-1), next_hi(-1),
+          end_published(false), n_pub(0),
           have_tile(false)
     {
         Us = a.with_shared ? a.rows[1] >> 4 : 0;
@@ -390,56 +390,68 @@ struct ItemWalk {
         if (lo >= P)
             lo = hi = -1;
     }
+    // Claimer: claims one more chunk and publishes it in the ring (with its group looked up
+    // in round-robin mode, so that the other roles need not go to global memory for it).
+    __device__ bool publish_one()
+    {
+        const int slot = n_pub % FF_CLAIMS;
+        const uint32_t par = (uint32_t)(n_pub / FF_CLAIMS) & 1u;
+        int lo, hi, sidx = 0;
+        Segment grp = sg;
+        claim(lo, hi);
+        if (lo >= 0 && a.round_robin) {
+            sidx = a.pair_first[lo / ntiles];
+            grp = a.seg[sidx];
+        }
+        if (!mbar_wait(ring.empty0 + 8u * slot, par ^ 1u, ring.abort_flag, ring.status))
+            return false;
+        int *e = ring.data + slot * FF_CLAIM_WORDS;
+        e[0] = lo;
+        e[1] = hi;
+        e[2] = sidx;
+        e[3] = grp.expert;
+        e[4] = grp.row0;
+        e[5] = grp.n;
+        e[6] = grp.first_seg;
+        __threadfence_block();
+        mbar_arrive(ring.full0 + 8u * slot);
+        ++n_pub;
+        if (lo < 0)
+            end_published = true;
+        return true;
+    }
     // Next chunk [lo, hi) of the routed work; false when none is left (or on abort).  In
-    // round-robin mode the chunk is one item and `grp` receives its group (the claimer looks
-    // it up once; the other roles take it from the ring instead of going to global memory).
-    // While plenty of work is left the claimer keeps one claim in flight beyond the one it
-    // hands out, so that the atomic's latency is not on the path of the weight stream.
+    // round-robin mode the chunk is one item and `grp` receives its group.  While plenty of
+    // work is left the claimer publishes one chunk beyond the one it is about to work on, so
+    // that every role knows its next item before it finishes the current one (near the end a
+    // chunk held in reserve would starve another CTA).
     __device__ bool acquire(int &lo, int &hi, Segment &grp, int &sidx)
     {
         const int slot = n_claims % FF_CLAIMS;
         const uint32_t par = (uint32_t)(n_claims / FF_CLAIMS) & 1u;
-        ++n_claims;
         int *e = ring.data + slot * FF_CLAIM_WORDS;
         if (claimer) {
-            if (primed) {
-                lo = next_lo;
-                hi = next_hi;
-            } else {
-                claim(lo, hi);
+            for (;;) {
+                const bool plenty =
+                    P - *reinterpret_cast<volatile int32_t *>(a.claim_counter) >
+                    4 * (long long)gridDim.x * (a.round_robin ? 1 : max_units);
+                if (end_published || n_pub >= n_claims + (plenty ? 2 : 1))
+                    break;
+                if (!publish_one())
+                    return false;
             }
-            // while plenty of work is left, the following claim is made now and consumed at
-            // the next call (near the end a claim held in reserve would starve another CTA)
-            primed = lo >= 0 &&
-                     P - *reinterpret_cast<volatile int32_t *>(a.claim_counter) > 4 * (long long)gridDim.x * (a.round_robin ? 1 : max_units);
-            if (primed)
-                claim(next_lo, next_hi);
-            sidx = 0;
-            if (lo >= 0 && a.round_robin) {
-                sidx = a.pair_first[lo / ntiles];
-                grp = a.seg[sidx];
-            }
-            if (!mbar_wait(ring.empty0 + 8u * slot, par ^ 1u, ring.abort_flag, ring.status))
-                return false;
-            e[0] = lo;
-            e[1] = hi;
-            e[2] = sidx;
-            e[3] = grp.expert;
-            e[4] = grp.row0;
-            e[5] = grp.n;
-            e[6] = grp.first_seg;
-            __threadfence_block();
-            mbar_arrive(ring.full0 + 8u * slot);
-        } else {
-            if (!mbar_wait(ring.full0 + 8u * slot, par, ring.abort_flag, ring.status))
-                return false;
-            lo = e[0];
-            hi = e[1];
-            sidx = e[2];
-            grp.expert = e[3];
-            grp.row0 = e[4];
-            grp.n = e[5];
-            grp.first_seg = e[6];
+        } else if (!mbar_wait(ring.full0 + 8u * slot, par, ring.abort_flag, ring.status)) {
+            return false;
+        }
+        ++n_claims;
+        lo = e[0];
+        hi = e[1];
+        sidx = e[2];
+        grp.expert = e[3];
+        grp.row0 = e[4];
+        grp.n = e[5];
+        grp.first_seg = e[6];
+        if (!claimer) {
             if (warp_wide)
                 __syncwarp();  // every lane has read the entry before it is released
             if (lead)
