@@ -113,18 +113,19 @@ def _full_size(name, B, gamma, n_rows, zipf=None):
     return check_layer_against_oracle(shape, w, x, B, gamma, rows=rows)
 
 
-@pytest.mark.parametrize("B,gamma", [(1, 0), (4, 1), (32, 3), (128, 4)])
+@pytest.mark.parametrize("B,gamma", [(1, 0), (4, 1), (32, 3), (128, 4), (1024, 3)])
 def test_full_size_qwen15_shape(B, gamma):
     _full_size("qwen1.5-moe-a2.7b", B, gamma, 6)
 
 
-@pytest.mark.parametrize("B,gamma,zipf", [(8, 2, None), (64, 4, 1.2)])
+@pytest.mark.parametrize("B,gamma,zipf", [(8, 2, None), (64, 4, 1.2), (256, 4, None)])
 def test_full_size_qwen2_57b_shape(B, gamma, zipf):
     _full_size("qwen2-57b-a14b", B, gamma, 3, zipf)
 
 
-def test_full_size_mixtral_shape():
-    _full_size("mixtral-8x7b", 16, 2, 3)
+@pytest.mark.parametrize("B,gamma", [(16, 2), (256, 4)])
+def test_full_size_mixtral_shape(B, gamma):
+    _full_size("mixtral-8x7b", B, gamma, 3)
 
 
 def test_full_size_deepseek_v3_shape():
