@@ -133,7 +133,9 @@ PlanView plan_view(char *ws, const Workspace &L)
 {
     return PlanView{reinterpret_cast<int32_t *>(ws + L.plan_header),
                     reinterpret_cast<Segment *>(ws + L.plan_seg),
-                    reinterpret_cast<int32_t *>(ws + L.plan_pairs)};
+                    reinterpret_cast<int32_t *>(ws + L.plan_pairs),
+                    reinterpret_cast<int32_t *>(ws + L.plan_done),
+                    reinterpret_cast<int32_t *>(ws + L.plan_done) + L.plan_done_shared_at};
 }
 
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
@@ -323,7 +325,8 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
         ~Arm() { g_probe_armed = false; }
     } arm;
     MOE_STAGE(MOE_STAGE_ROUTER_LOGITS,
-              launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s));
+              launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s,
+                                   plan_view(base, L).done_shared, max_shared_segments(T)));
     MOE_STAGE(MOE_STAGE_ROUTE_TOPK, launch_route_topk(*cfg, logits, T, topk_idx, topk_w, s));
     // the grouping kernel also writes the FFN segment plan (one launch fewer)
     const PlanView plan = plan_view(base, L);

@@ -33,7 +33,14 @@ struct PlanView {
     int32_t *header;      // written by the plan; [2], [3] advanced by the FFN kernels
     Segment *seg;         // capacity max_segments()
     int32_t *pair_first;  // plan index of every pair's first segment, capacity max_segments()
+    // Progress of the gate/up pass, read by the down pass: 16-row units of h written so far
+    // (counted once per epilogue warp) for every routed segment [max_segments()] and for
+    // every 128-row segment of the shared expert [max_shared_segments()].
+    int32_t *done_routed;
+    int32_t *done_shared;
 };
+
+__host__ __device__ inline int max_shared_segments(int T) { return (T + SEG_TOKENS - 1) / SEG_TOKENS; }
 
 __host__ __device__ inline int max_segments(int E, int A) { return E + A / SEG_TOKENS + 1; }
 
@@ -55,6 +62,8 @@ struct Workspace {
     size_t plan_header;   // i32 [PLAN_HEADER_INTS]
     size_t plan_seg;      // Segment[max_segments]
     size_t plan_pairs;    // i32 [max_segments]
+    size_t plan_done;     // i32 [max_segments + max_shared_segments]
+    size_t plan_done_shared_at;  // index of the shared expert's counters inside plan_done
     size_t x_sorted;      // bf16 [A, H]      token rows in sorted order
     size_t h;             // bf16 [A, I]      SwiGLU intermediate, sorted order
     size_t h_shared;      // bf16 [T, I_s]
@@ -93,6 +102,8 @@ inline Workspace workspace_layout(const moe_config_t &c, int T)
     w.plan_header = take(PLAN_HEADER_INTS * 4);
     w.plan_seg = take(sizeof(Segment) * (size_t)max_segments((int)E, (int)A));
     w.plan_pairs = take(4 * (size_t)max_segments((int)E, (int)A));
+    w.plan_done = take(4 * ((size_t)max_segments((int)E, (int)A) + max_shared_segments(T)));
+    w.plan_done_shared_at = (size_t)max_segments((int)E, (int)A);
     w.x_sorted = take(A * H * 2);
     w.h = take(A * (size_t)c.inter * 2);
     w.h_shared = take((size_t)T * c.shared_inter * 2);
@@ -109,9 +120,12 @@ struct LaunchCounter {
     int n = 0;
 };
 
+// zero / zero_n: ints this kernel clears before any later kernel of the call may start (the
+// shared expert's progress counters), or null
 cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
                                  const __nv_bfloat16 *x, int T, float *logits,
-                                 float *shared_scale, cudaStream_t s);
+                                 float *shared_scale, cudaStream_t s, int32_t *zero = nullptr,
+                                 int zero_n = 0);
 cudaError_t launch_route_topk(const moe_config_t &c, const float *logits, int T, int32_t *idx,
                               float *wts, cudaStream_t s);
 cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int32_t *counts,

@@ -68,6 +68,8 @@ struct FfnArgs {
     const Segment *seg;
     const int32_t *pair_first;   // plan index of every pair's first segment
     int32_t *claim_counter;      // grid-wide: next unclaimed routed position / item of this pass
+    int32_t *done[2];            // per segment of each group kind: 16-column units of h finished
+                                 // by the gate/up pass, summed over its four epilogue warps
     int round_robin;             // routed work dealt as (pair, tile) items instead of ranges
     int32_t *status;
     int T;             // token rows (the shared expert's group)
@@ -149,6 +151,36 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity))
                 return true;
+        if (*abort_flag)
+            return false;
+        if (global_ns() - t0 > FF_WAIT_NS) {
+            *abort_flag = 1;
+            atomicExch(status, 1);
+            return false;
+        }
+    }
+}
+
+// Bounded wait until the progress counter at p has reached `target` (acquire: what the
+// writers stored before their adds is visible afterwards).  Same failure handling as mbar_wait.
+__device__ __forceinline__ bool counter_wait(const int32_t *p, int target, volatile int *abort_flag,
+                                             int32_t *status)
+{
+    auto reached = [&]() {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+        return v >= target;
+    };
+    if (reached())
+        return true;
+    const uint64_t t0 = global_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 16; ++i) {
+            if (reached())
+                return true;
+            __nanosleep(100);
+        }
         if (*abort_flag)
             return false;
         if (global_ns() - t0 > FF_WAIT_NS) {
@@ -276,6 +308,7 @@ struct Item {
     int row0;    // first token row (sorted row for routed groups, token for the shared expert)
     int n;       // token rows, 1..FF_SEG
     int role;    // 0 single, 1 first of a pair, 2 second of a pair (shares the first's tile)
+    int seg;     // index of the segment's progress counter (plan index; shared: segment number)
     int w_once;  // the tile's weights are read by this item (or pair) only
     int k0, k1;  // reduction range [k0, k1)
     long long out_off;  // element offset of this item's output plane (k chunk) in out[grp]
@@ -328,7 +361,7 @@ struct ItemWalk {
     Segment sg;
     int g_nseg, g_u_end;
     bool have_tile;
-    int t_grp, t_expert, t_u0, t_h, t_row0, t_n, t_s, t_s_end;
+    int t_grp, t_expert, t_u0, t_h, t_row0, t_n, t_s, t_s_end, t_seg0;
     bool t_once;  // the tile's weights are read by this pass over it only
     int t_k0, t_k1;
     long long t_out_off;
@@ -473,6 +506,7 @@ struct ItemWalk {
                     it.n = min(FF_SEG, t_n - t_s * FF_SEG);
                     // segments 2q and 2q+1 of a tile form a pair
                     it.role = (t_s & 1) ? 2 : (t_s + 1 < t_s_end ? 1 : 0);
+                    it.seg = t_seg0 + t_s;
                     it.w_once = t_once;
                     it.k0 = t_k0;
                     it.k1 = t_k1;
@@ -493,6 +527,7 @@ struct ItemWalk {
                 t_grp = 1;
                 t_expert = 0;
                 t_row0 = 0;
+                t_seg0 = 0;
                 t_n = a.T;
                 t_s = 2 * q;
                 t_s_end = min(nseg_s, 2 * q + 2);
@@ -520,6 +555,7 @@ struct ItemWalk {
                     t_grp = 0;
                     t_expert = sg.expert;
                     t_row0 = sg.row0;
+                    t_seg0 = sg.first_seg;
                     t_n = sg.n;
                     t_s = sidx - sg.first_seg;
                     t_s_end = min(g_nseg, t_s + 2);
@@ -551,6 +587,7 @@ struct ItemWalk {
                 t_expert = sg.expert;
                 t_u0 = u;
                 t_row0 = sg.row0;
+                t_seg0 = sg.first_seg;
                 t_n = sg.n;
                 t_s = 0;
                 t_s_end = g_nseg;
@@ -750,11 +787,11 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
     } else if (warp == 2) {
         // ---------------- token-operand producer ----------------
         if (lane == 0) {
-            // down pass: h is written by the preceding kernel
-            if (!GATED)
-                griddep_wait();
+            // down pass: h is written by the preceding kernel, which may still be running; a
+            // segment's rows are fetched once its progress counter says they are complete
             ItemWalk walk(args, claims, false, true, false, !GATED);
             XRingWalk ring(args.x_units);
+            int seen[2] = {-1, -1};  // (group, segment) keys last found complete
             const uint64_t pol_keep = l2_policy_evict_last();
             int released = 0;          // entries known to have been consumed
             int v_cur = 0, v_rel = 0;  // virtual unit positions: issued up to / released up to
@@ -768,6 +805,23 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 if (nsub == 2 && !walk.next(it2))
                     break;  // cannot happen: a first is always followed by its second
                 const int K = it.k1;
+                if (!GATED) {
+                    for (int sub = 0; ok && sub < nsub; ++sub) {
+                        const Item &cur = sub ? it2 : it;
+                        const int key = (cur.grp << 30) | cur.seg;
+                        if (key == seen[0] || key == seen[1])
+                            continue;
+                        // every epilogue warp of the gate/up pass counts the 16-column units
+                        // of h it has finished for the segment
+                        ok = counter_wait(args.done[cur.grp] + cur.seg, args.K[cur.grp] >> 2, abortp,
+                                          args.status);
+                        seen[sub] = key;
+                    }
+                    if (!ok)
+                        break;
+                    // rows written through the generic proxy, read below by the async proxy
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
+                }
                 for (int k0 = it.k0; ok && k0 < K; k0 += 64 * kb) {
                     const int nbox = min(kb, (K - k0 + 63) >> 6);
                     for (int sub = 0; sub < nsub; ++sub) {
@@ -817,6 +871,8 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             }
             if (!walk.synced)
                 walk.sync(true);
+            if (!GATED)
+                griddep_wait();  // no kernel of the chain completes before its predecessor
             if (!ok) {
                 const uint64_t t0 = global_ns();
                 while (global_ns() - t0 < 1000000ull) {
@@ -912,10 +968,8 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
         }
     } else {
         // ---------------- epilogue (warps 3..6) ----------------
-        // down pass: everything this kernel writes or reads besides weights belongs to the
-        // layer call in flight, so it waits for the preceding kernel first
-        if (!GATED)
-            griddep_wait();
+        // down pass: its outputs are read by nothing older than this call's combine, so the
+        // stores need not wait for the preceding kernel (the token producer does, per segment)
         const int quarter = warp & 3;  // TMEM lanes 32*quarter .. +31 belong to this warp
         ItemWalk walk(args, claims, false, lane == 0, true, !GATED);
         int n_items = 0;
@@ -967,9 +1021,17 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 }
             }
             tc_fence_before();
+            if (GATED)  // the down pass fetches these rows with TMA (async proxy)
+                asm volatile("fence.proxy.async.global;" ::: "memory");
             __syncwarp();
-            if (lane == 0)
+            if (lane == 0) {
                 mbar_arrive(acc_empty(buf));
+                if (GATED) {
+                    // publish: this warp's part of the tile is in h
+                    __threadfence();
+                    atomicAdd(args.done[it.grp] + it.seg, it.h >> 4);
+                }
+            }
         }
         if (!walk.synced)
             walk.sync(true);
@@ -1198,6 +1260,8 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
     a.seg = plan.seg;
     a.pair_first = plan.pair_first;
     a.claim_counter = plan.header + 2;
+    a.done[0] = plan.done_routed;
+    a.done[1] = plan.done_shared;
     a.round_robin = use_round_robin(c, T, c.inter, c.hidden, a.max_tile, ffn_grid()) ? 1 : 0;
     a.status = status;
     a.T = T;
@@ -1248,6 +1312,8 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
     a.seg = plan.seg;
     a.pair_first = plan.pair_first;
     a.claim_counter = plan.header + 3;
+    a.done[0] = plan.done_routed;
+    a.done[1] = plan.done_shared;
     a.round_robin = use_round_robin(c, T, c.hidden, c.inter, a.max_tile, ffn_grid()) ? 1 : 0;
     a.status = status;
     a.T = T;

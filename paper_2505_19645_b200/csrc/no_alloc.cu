@@ -54,6 +54,8 @@ static Workspace static_scratch_layout(const moe_config_t &c, int T)
     w.plan_header = take(PLAN_HEADER_INTS * 4);
     w.plan_seg = take(sizeof(Segment) * (size_t)max_segments(c.n_experts, (int)A));
     w.plan_pairs = take(4 * (size_t)max_segments(c.n_experts, (int)A));
+    w.plan_done = take(4 * ((size_t)max_segments(c.n_experts, (int)A) + max_shared_segments(T)));
+    w.plan_done_shared_at = (size_t)max_segments(c.n_experts, (int)A);
     w.x_sorted = take(A * (size_t)c.hidden * 2);
     w.h = take(A * (size_t)c.inter * 2);
     w.h_shared = take((size_t)T * c.shared_inter * 2);
@@ -91,9 +93,9 @@ moe_status_t moe_grouped_swiglu_static(const moe_config_t *cfg, const moe_weight
     if ((st = static_scratch_address(&scratch)) != MOE_OK)
         return st;
     int launches = 0;
-    // The plan kernel, first in the sequence, clears the status word and rewrites the whole
-    // plan; h is fully written by the gate/up pass before the down pass reads it.  Nothing
-    // else in the array has to start at zero.
+    // The plan kernel, first in the sequence, clears the status word and the progress
+    // counters and rewrites the whole plan; the down pass reads a segment of h only once the
+    // gate/up pass has counted it complete.  Nothing else in the array has to start at zero.
     return run_ffn(*cfg, *w, static_cast<const __nv_bfloat16 *>(x), T, offsets, perm,
                    static_cast<__nv_bfloat16 *>(y), static_cast<__nv_bfloat16 *>(shared_y), scratch,
                    L, static_cast<cudaStream_t>(stream), launches);

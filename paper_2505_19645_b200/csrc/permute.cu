@@ -69,8 +69,10 @@ __device__ void build_plan(const int *cnt_sh, const int *off_sh, int *scan, int 
         sg.row0 = row0;
         sg.n = cnt;
         sg.first_seg = first;
-        for (int i = 0; i < nseg; ++i)
+        for (int i = 0; i < nseg; ++i) {
             plan.seg[first + i] = sg;
+            plan.done_routed[first + i] = 0;
+        }
     }
     if (tid == 0) {
         plan.header[0] = *total;
@@ -214,7 +216,7 @@ cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int
 
 // Stand-alone plan (moe_grouped_swiglu gets its offsets from the caller).
 __global__ void __launch_bounds__(MOE_MAX_EXPERTS)
-plan_kernel(const int32_t *__restrict__ offsets, int E, int32_t *__restrict__ status, PlanView plan)
+plan_kernel(const int32_t *__restrict__ offsets, int E, int T, int32_t *__restrict__ status, PlanView plan)
 {
     __shared__ int cnt[MOE_MAX_EXPERTS];
     __shared__ int offs[MOE_MAX_EXPERTS];
@@ -222,6 +224,12 @@ plan_kernel(const int32_t *__restrict__ offsets, int E, int32_t *__restrict__ st
     __shared__ int tmp[MOE_MAX_EXPERTS];
     __shared__ int total;
     griddep_wait();
+    // first kernel of the stand-alone FFN call: the shared expert's progress counters must be
+    // clear before the gate/up pass, which may start right away, counts on them
+    for (int i = threadIdx.x; i < max_shared_segments(T); i += blockDim.x)
+        plan.done_shared[i] = 0;
+    __threadfence();
+    __syncthreads();
     griddep_launch();
     const int tid = threadIdx.x;
     int row0 = 0, n = 0;
@@ -238,8 +246,7 @@ plan_kernel(const int32_t *__restrict__ offsets, int E, int32_t *__restrict__ st
 cudaError_t launch_plan(const moe_config_t &c, int T, const int32_t *offsets, int32_t *status,
                         PlanView plan, cudaStream_t s)
 {
-    (void)T;
-    return launch_pdl(plan_kernel, dim3(1), dim3(MOE_MAX_EXPERTS), 0, s, offsets, c.n_experts, status,
+    return launch_pdl(plan_kernel, dim3(1), dim3(MOE_MAX_EXPERTS), 0, s, offsets, c.n_experts, T, status,
                       plan);
 }
 

@@ -64,11 +64,18 @@ __global__ void __launch_bounds__(RL_WARPS_FOR(NCH) * 32)
 router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ w_router,
                      const float *__restrict__ bias, const __nv_bfloat16 *__restrict__ w_sg,
                      int T, int H, int E, int n_rows, float *__restrict__ logits,
-                     float *__restrict__ shared_scale)
+                     float *__restrict__ shared_scale, int32_t *__restrict__ zero, int zero_n)
 {
     constexpr int RL_WARPS = RL_WARPS_FOR(NCH);
     __shared__ float part[RL_WARPS][NCH][4][32];
     griddep_wait();    // first kernel of a layer call: everything older is complete from here on
+    if (zero != nullptr && blockIdx.x == 0 && blockIdx.y == 0) {
+        // counters that a later kernel of this call updates before the plan kernel has run
+        for (int i = threadIdx.x; i < zero_n; i += blockDim.x)
+            zero[i] = 0;
+        __threadfence();
+        __syncthreads();
+    }
     griddep_launch();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;
@@ -152,7 +159,7 @@ router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restric
 
 cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
                                  const __nv_bfloat16 *x, int T, float *logits,
-                                 float *shared_scale, cudaStream_t s)
+                                 float *shared_scale, cudaStream_t s, int32_t *zero, int zero_n)
 {
     const bool gate_row = shared_scale != nullptr && c.shared_gate && c.shared_inter > 0;
     const int n_rows = c.n_experts + (gate_row ? 1 : 0);
@@ -165,7 +172,8 @@ cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
     const __nv_bfloat16 *w_sg = static_cast<const __nv_bfloat16 *>(w.w_shared_gate);
 #define MOE_RL_LAUNCH(N)                                                                    \
     err = launch_pdl(router_logits_kernel<N>, grid, dim3(RL_WARPS_FOR(N) * 32), 0, s, x, w.w_router,    \
-                     w.router_bias, w_sg, T, c.hidden, c.n_experts, n_rows, logits, shared_scale)
+                     w.router_bias, w_sg, T, c.hidden, c.n_experts, n_rows, logits, shared_scale, zero,  \
+                     zero_n)
     cudaError_t err = cudaSuccess;
     switch (nch) {
     case 1: MOE_RL_LAUNCH(1); break;
