@@ -141,7 +141,7 @@ PlanView plan_view(char *ws, const Workspace &L)
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
                      const int32_t *offsets, const int32_t *perm, __nv_bfloat16 *y,
                      __nv_bfloat16 *shared_y, char *ws, const Workspace &L, cudaStream_t s,
-                     int &launches, bool plan_ready, int shared_parts)
+                     int &launches, bool plan_ready, int shared_parts, int routed_parts)
 {
     const bool with_shared = shared_y != nullptr && c.shared_inter > 0;
     const PlanView plan = plan_view(ws, L);
@@ -155,7 +155,8 @@ moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_b
     MOE_STAGE(MOE_STAGE_GATE_UP,
               launch_ffn_gateup(c, w, x, xs, T, plan, with_shared, h, hs, status, s));
     MOE_STAGE(MOE_STAGE_DOWN,
-              launch_ffn_down(c, w, T, plan, with_shared, h, hs, y, shared_y, shared_parts, status, s));
+              launch_ffn_down(c, w, T, plan, with_shared, h, hs, y, shared_y, shared_parts,
+                              routed_parts, status, s));
     return MOE_OK;
 }
 
@@ -271,7 +272,7 @@ moe_status_t moe_combine(const moe_config_t *cfg, const void *y, const int32_t *
     if ((st = check_device()) != MOE_OK)
         return st;
     int launches = 0;
-    MOE_TRY_LAUNCH(launch_combine(*cfg, static_cast<const __nv_bfloat16 *>(y), inv_perm, topk_w,
+    MOE_TRY_LAUNCH(launch_combine(*cfg, static_cast<const __nv_bfloat16 *>(y), 1, inv_perm, topk_w,
                                   static_cast<const __nv_bfloat16 *>(shared_y), 1, shared_scale, T,
                                   static_cast<__nv_bfloat16 *>(out),
                                   static_cast<cudaStream_t>(stream)));
@@ -334,11 +335,13 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
               launch_permute(*cfg, topk_idx, T, counts, offsets, perm, inv_perm, active, n_active, s,
                              &plan, reinterpret_cast<int32_t *>(base + L.status)));
     const int shared_parts = has_shared ? shared_down_parts(*cfg) : 1;
-    st = run_ffn(*cfg, *w, xb, T, offsets, perm, y, ys, base, L, s, launches, true, shared_parts);
+    const int routed_parts = routed_down_parts(*cfg, T);
+    st = run_ffn(*cfg, *w, xb, T, offsets, perm, y, ys, base, L, s, launches, true, shared_parts,
+                 routed_parts);
     if (st != MOE_OK)
         return st;
     MOE_STAGE(MOE_STAGE_COMBINE,
-              launch_combine(*cfg, y, inv_perm, topk_w, ys, shared_parts, gated ? shared_scale : nullptr, T,
+              launch_combine(*cfg, y, routed_parts, inv_perm, topk_w, ys, shared_parts, gated ? shared_scale : nullptr, T,
                              static_cast<__nv_bfloat16 *>(out), s));
     g_last_launches = launches;
 

@@ -1,4 +1,5 @@
-// Gate-weighted combine: out[t] = sum_j w[t,j] * y[inv_perm[t*K+j]] + s[t] * shared_y[t].
+// Gate-weighted combine: out[t] = sum_j w[t,j] * y[inv_perm[t*K+j]] + s[t] * shared_y[t]
+// (y and shared_y may arrive as partial planes, one per k chunk of the down projection).
 // Gather form (each output row is summed in slot order by one owner), so the result does
 // not depend on scheduling; 128-bit loads and stores.
 #include "common.cuh"
@@ -8,7 +9,8 @@ namespace moe {
 constexpr int CB_THREADS = 256;
 
 __global__ void __launch_bounds__(CB_THREADS)
-combine_kernel(const __nv_bfloat16 *__restrict__ y, const int32_t *__restrict__ inv_perm,
+combine_kernel(const __nv_bfloat16 *__restrict__ y, int routed_parts,
+               const int32_t *__restrict__ inv_perm,
                const float *__restrict__ topk_w, const __nv_bfloat16 *__restrict__ shared_y,
                int shared_parts, const float *__restrict__ shared_scale, int T, int H, int k,
                __nv_bfloat16 *__restrict__ out)
@@ -31,27 +33,30 @@ combine_kernel(const __nv_bfloat16 *__restrict__ y, const int32_t *__restrict__ 
             wts[j] = j < k ? topk_w[(size_t)t * k + j] : 0.f;
         }
         const float s = shared_y && shared_scale ? shared_scale[t] : 1.0f;
-        uint4 v[MOE_MAX_TOPK];
-#pragma unroll
-        for (int j = 0; j < MOE_MAX_TOPK; ++j)
-            if (j < k)
-                v[j] = *reinterpret_cast<const uint4 *>(y + (size_t)rows[j] * H + h);
         float acc[8];
 #pragma unroll
         for (int q = 0; q < 8; ++q)
             acc[q] = 0.f;
+        for (int part = 0; part < routed_parts; ++part) {
+            const __nv_bfloat16 *yp = y + (size_t)part * T * k * H;
+            uint4 v[MOE_MAX_TOPK];
 #pragma unroll
-        for (int j = 0; j < MOE_MAX_TOPK; ++j) {
-            if (j < k) {
-                const float w = wts[j];
-                acc[0] = fmaf(w, bf16_lo(v[j].x), acc[0]);
-                acc[1] = fmaf(w, bf16_hi(v[j].x), acc[1]);
-                acc[2] = fmaf(w, bf16_lo(v[j].y), acc[2]);
-                acc[3] = fmaf(w, bf16_hi(v[j].y), acc[3]);
-                acc[4] = fmaf(w, bf16_lo(v[j].z), acc[4]);
-                acc[5] = fmaf(w, bf16_hi(v[j].z), acc[5]);
-                acc[6] = fmaf(w, bf16_lo(v[j].w), acc[6]);
-                acc[7] = fmaf(w, bf16_hi(v[j].w), acc[7]);
+            for (int j = 0; j < MOE_MAX_TOPK; ++j)
+                if (j < k)
+                    v[j] = *reinterpret_cast<const uint4 *>(yp + (size_t)rows[j] * H + h);
+#pragma unroll
+            for (int j = 0; j < MOE_MAX_TOPK; ++j) {
+                if (j < k) {
+                    const float w = wts[j];
+                    acc[0] = fmaf(w, bf16_lo(v[j].x), acc[0]);
+                    acc[1] = fmaf(w, bf16_hi(v[j].x), acc[1]);
+                    acc[2] = fmaf(w, bf16_lo(v[j].y), acc[2]);
+                    acc[3] = fmaf(w, bf16_hi(v[j].y), acc[3]);
+                    acc[4] = fmaf(w, bf16_lo(v[j].z), acc[4]);
+                    acc[5] = fmaf(w, bf16_hi(v[j].z), acc[5]);
+                    acc[6] = fmaf(w, bf16_lo(v[j].w), acc[6]);
+                    acc[7] = fmaf(w, bf16_hi(v[j].w), acc[7]);
+                }
             }
         }
         if (shared_y) {
@@ -82,8 +87,9 @@ combine_kernel(const __nv_bfloat16 *__restrict__ y, const int32_t *__restrict__ 
     }
 }
 
-cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, const int32_t *inv_perm,
-                           const float *topk_w, const __nv_bfloat16 *shared_y, int shared_parts,
+cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, int routed_parts,
+                           const int32_t *inv_perm, const float *topk_w,
+                           const __nv_bfloat16 *shared_y, int shared_parts,
                            const float *shared_scale, int T, __nv_bfloat16 *out, cudaStream_t s)
 {
     const size_t total = (size_t)T * (c.hidden >> 3);
@@ -91,8 +97,8 @@ cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, const 
     const size_t cap = (size_t)sm_count() * 8;
     if (blocks > cap)
         blocks = cap;
-    return launch_pdl(combine_kernel, dim3((unsigned)blocks), dim3(CB_THREADS), 0, s, y, inv_perm,
-                      topk_w, shared_y, shared_parts, shared_scale, T, c.hidden, c.top_k, out);
+    return launch_pdl(combine_kernel, dim3((unsigned)blocks), dim3(CB_THREADS), 0, s, y, routed_parts,
+                      inv_perm, topk_w, shared_y, shared_parts, shared_scale, T, c.hidden, c.top_k, out);
 }
 
 }  // namespace moe

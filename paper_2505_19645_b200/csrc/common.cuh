@@ -77,6 +77,10 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // k chunks the shared expert's down projection is split into inside moe_verify_layer (each
 // chunk is a work unit of its own and writes a partial [T,H] plane that the combine step sums)
 int shared_down_parts(const moe_config_t &c);
+// k chunks of the routed groups' down projection for T tokens (1 above a few tokens)
+constexpr int ROUTED_SPLIT_MAX_TOKENS = 16;
+constexpr int ROUTED_SPLIT_MAX_PARTS = 8;
+int routed_down_parts(const moe_config_t &c, int T);
 
 inline Workspace workspace_layout(const moe_config_t &c, int T)
 {
@@ -107,7 +111,11 @@ inline Workspace workspace_layout(const moe_config_t &c, int T)
     w.x_sorted = take(A * H * 2);
     w.h = take(A * (size_t)c.inter * 2);
     w.h_shared = take((size_t)T * c.shared_inter * 2);
-    w.y = take(A * H * 2);
+    // y: [A,H], or for few tokens up to ROUTED_SPLIT_MAX_PARTS partial planes of it
+    const size_t A_small = A < (size_t)ROUTED_SPLIT_MAX_TOKENS * c.top_k
+                               ? A : (size_t)ROUTED_SPLIT_MAX_TOKENS * c.top_k;
+    const size_t y_rows = A > ROUTED_SPLIT_MAX_PARTS * A_small ? A : ROUTED_SPLIT_MAX_PARTS * A_small;
+    w.y = take(y_rows * H * 2);
     w.y_shared = take((size_t)T * H * 2 * shared_down_parts(c));
     w.total = off;
     return w;
@@ -144,13 +152,16 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
 cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T, PlanView plan,
                             bool with_shared, const __nv_bfloat16 *h, const __nv_bfloat16 *h_shared,
                             __nv_bfloat16 *y, __nv_bfloat16 *y_shared, int shared_parts,
+                            int routed_parts,
                             int32_t *status, cudaStream_t s);
 // token rows in sorted order (the token operand of the routed gate/up tiles)
 cudaError_t launch_gather_rows(const moe_config_t &c, const __nv_bfloat16 *x, const int32_t *perm,
                                int T, __nv_bfloat16 *x_sorted, cudaStream_t s);
-// shared_y may hold `shared_parts` partial planes [T,H] (k chunks of the down pass), summed here
-cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, const int32_t *inv_perm,
-                           const float *topk_w, const __nv_bfloat16 *shared_y, int shared_parts,
+// y and shared_y may hold `routed_parts` / `shared_parts` partial planes ([A,H] / [T,H]: k
+// chunks of the down pass), summed here
+cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, int routed_parts,
+                           const int32_t *inv_perm, const float *topk_w,
+                           const __nv_bfloat16 *shared_y, int shared_parts,
                            const float *shared_scale, int T, __nv_bfloat16 *out, cudaStream_t s);
 
 int sm_count();
@@ -167,7 +178,8 @@ PlanView plan_view(char *ws, const Workspace &L);
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
                      const int32_t *offsets, const int32_t *perm, __nv_bfloat16 *y,
                      __nv_bfloat16 *shared_y, char *ws, const Workspace &L, cudaStream_t s,
-                     int &launches, bool plan_ready = false, int shared_parts = 1);
+                     int &launches, bool plan_ready = false, int shared_parts = 1,
+                     int routed_parts = 1);
 
 // ---------------------------------------------------------------------------------------
 // Device helpers.

@@ -79,6 +79,9 @@ struct FfnArgs {
                          // to out[1] + s * shared_part_stride
     int shared_kchunk;   // multiple of 128
     long long shared_part_stride;  // elements
+    int routed_ksplit;   // the same for the routed groups (round-robin mode of the down pass only)
+    int routed_kchunk;
+    long long routed_part_stride;
     int shared_tiles;  // tiles of the shared expert's rows; (tile, segment pair) units are dealt
                        // round-robin to the CTAs; the first (units % tiles) tiles have one
                        // 16-row unit more
@@ -406,7 +409,8 @@ struct ItemWalk {
         if (wait)
             griddep_wait();
         nseg_total = a.plan_header[0];
-        P = a.round_robin ? (long long)a.plan_header[1] * ntiles : (long long)nseg_total * R0;
+        P = a.round_robin ? (long long)a.plan_header[1] * ntiles * a.routed_ksplit
+                          : (long long)nseg_total * R0;
         synced = true;
     }
     // Claims the next chunk from the grid-wide counter (claimer only).
@@ -433,7 +437,7 @@ struct ItemWalk {
         Segment grp = sg;
         claim(lo, hi);
         if (lo >= 0 && a.round_robin) {
-            sidx = a.pair_first[lo / ntiles];
+            sidx = a.pair_first[lo / (ntiles * a.routed_ksplit)];
             grp = a.seg[sidx];
         }
         if (!mbar_wait(ring.empty0 + 8u * slot, par ^ 1u, ring.abort_flag, ring.status))
@@ -547,8 +551,9 @@ struct ItemWalk {
                     return false;
                 }
                 if (a.round_robin) {
-                    // one (pair, tile) item
-                    const int tile = lo % ntiles;
+                    // one (pair, tile, k chunk) item
+                    const int chunk = lo % a.routed_ksplit;
+                    const int tile = (lo / a.routed_ksplit) % ntiles;
                     g_nseg = (sg.n + FF_SEG - 1) / FF_SEG;
                     t_u0 = tile * max_units;
                     t_h = min(max_units, R0 - t_u0);
@@ -560,9 +565,9 @@ struct ItemWalk {
                     t_s = sidx - sg.first_seg;
                     t_s_end = min(g_nseg, t_s + 2);
                     t_once = g_nseg <= 2;
-                    t_k0 = 0;
-                    t_k1 = a.K[0];
-                    t_out_off = 0;
+                    t_k0 = chunk * a.routed_kchunk;
+                    t_k1 = min(a.K[0], t_k0 + a.routed_kchunk);
+                    t_out_off = chunk * a.routed_part_stride;
                     have_tile = true;
                     continue;
                 }
@@ -1263,10 +1268,36 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
     a.done[0] = plan.done_routed;
     a.done[1] = plan.done_shared;
     a.round_robin = use_round_robin(c, T, c.inter, c.hidden, a.max_tile, ffn_grid()) ? 1 : 0;
+    a.routed_ksplit = 1;
+    a.routed_kchunk = c.hidden;
     a.status = status;
     a.T = T;
     a.with_shared = with_shared ? 1 : 0;
     return launch_ffn<true>(a, maps, s);
+}
+
+// Length of a k chunk when K is cut into about `parts` pieces (a multiple of the 128-column
+// weight slot), and the number of non-empty chunks that length gives.
+static int split_chunk(int K, int parts) { return ((K + parts - 1) / parts + 127) / 128 * 128; }
+static int split_parts(int K, int parts) { return (K + split_chunk(K, parts) - 1) / split_chunk(K, parts); }
+
+// k chunks of the routed groups' down projection.  With few tokens the pass has fewer
+// (pair, tile) items than CTAs and one SM cannot pull a tile faster than a fraction of what
+// HBM delivers, so the reduction is cut until about three items per CTA exist; each chunk
+// writes its own plane of y and the combine adds the planes.  Only for T <= 16 (the planes
+// must fit the workspace) and only where the pass deals single items.
+int routed_down_parts(const moe_config_t &c, int T)
+{
+    if (T > ROUTED_SPLIT_MAX_TOKENS || !use_round_robin(c, T, c.hidden, c.inter, 256, ffn_grid()))
+        return 1;
+    const double items = ceil(expected_active_experts(c.n_experts, c.top_k, T)) * ((c.hidden + 255) / 256);
+    int parts = (int)ceil(3.0 * ffn_grid() / items);
+    const int cap = c.inter / 1024;  // chunks below half a megabyte cost more than they level
+    if (parts > cap)
+        parts = cap;
+    if (parts > ROUTED_SPLIT_MAX_PARTS)
+        parts = ROUTED_SPLIT_MAX_PARTS;
+    return parts < 1 ? 1 : split_parts(c.inter, parts);
 }
 
 int shared_down_parts(const moe_config_t &c)
@@ -1274,13 +1305,13 @@ int shared_down_parts(const moe_config_t &c)
     if (c.shared_inter < 2 * c.inter)
         return 1;
     const int s = c.shared_inter / c.inter;
-    return s > 8 ? 8 : s;
+    return split_parts(c.shared_inter, s > 8 ? 8 : s);
 }
 
 cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T, PlanView plan,
                             bool with_shared, const __nv_bfloat16 *h, const __nv_bfloat16 *h_shared,
                             __nv_bfloat16 *y, __nv_bfloat16 *y_shared, int shared_parts,
-                            int32_t *status, cudaStream_t s)
+                            int routed_parts, int32_t *status, cudaStream_t s)
 {
     const uint64_t A = (uint64_t)T * c.top_k, H = c.hidden, E = c.n_experts;
     FfnArgs a{};
@@ -1289,8 +1320,7 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
     a.K[1] = c.shared_inter;
     a.max_tile = 256;
     a.shared_ksplit = with_shared ? shared_parts : 1;
-    a.shared_kchunk = with_shared ? ((c.shared_inter + a.shared_ksplit - 1) / a.shared_ksplit + 127) / 128 * 128
-                                  : 128;
+    a.shared_kchunk = with_shared ? split_chunk(c.shared_inter, a.shared_ksplit) : 128;
     a.shared_part_stride = (long long)T * c.hidden;
     a.shared_tiles = with_shared ? shared_tile_count(c, T, c.hidden, c.hidden, c.inter, c.shared_inter,
                                                      a.shared_ksplit, 128, 256, ffn_grid())
@@ -1315,6 +1345,14 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
     a.done[0] = plan.done_routed;
     a.done[1] = plan.done_shared;
     a.round_robin = use_round_robin(c, T, c.hidden, c.inter, a.max_tile, ffn_grid()) ? 1 : 0;
+    if (routed_parts > 1 && !a.round_robin)
+        return cudaErrorInvalidValue;  // planes exist only where single items are dealt
+    a.routed_ksplit = routed_parts;
+    a.routed_kchunk = split_chunk(c.inter, routed_parts);
+    if ((long long)(routed_parts - 1) * a.routed_kchunk >= c.inter ||
+        (with_shared && (long long)(a.shared_ksplit - 1) * a.shared_kchunk >= c.shared_inter))
+        return cudaErrorInvalidValue;  // an empty chunk would leave its plane unwritten
+    a.routed_part_stride = (long long)A * c.hidden;
     a.status = status;
     a.T = T;
     a.with_shared = with_shared ? 1 : 0;
