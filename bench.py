@@ -237,7 +237,7 @@ def run_reference(args):
     rank, _, world = replicas.env_world()
     if rank != 0:
         return 0
-    shape = wl.CONFIGS[args.config]
+    shape = variant_shape(args)
     T = args.B * (args.gamma + 1)
     w = wl.make_weights(shape, wl.config_seed(args.config), "cpu")
     x = wl.make_tokens(shape, T, wl.point_seed(args.config, args.B, args.gamma), "cpu")
@@ -272,7 +272,24 @@ def run_reference(args):
 
 def workload_name(args):
     return "%s-shaped MoE FFN layer, B=%d, gamma=%d (T=%d tokens)" % (
-        args.config, args.B, args.gamma, args.B * (args.gamma + 1))
+        variant_shape(args).name, args.B, args.gamma, args.B * (args.gamma + 1))
+
+
+def variant_shape(args):
+    """The config's layer shape, or its --top-k / --dense-contrast variant."""
+    shape = wl.CONFIGS[args.config]
+    if args.dense_contrast:
+        return wl.dense_contrast(shape)
+    if args.top_k is not None:
+        return wl.with_top_k(shape, args.top_k)
+    return shape
+
+
+def sweep_grid(args):
+    """(batch sizes, draft lengths) of the sweep: the config's own grid or the sparsity grid."""
+    if args.grid == "sparsity":
+        return wl.SPARSITY_BATCHES, wl.SPARSITY_GAMMAS
+    return wl.GRIDS[args.config]
 
 
 def main():
@@ -285,6 +302,12 @@ def main():
     ap.add_argument("--B", type=int, default=DEFAULT_B)
     ap.add_argument("--gamma", type=int, default=DEFAULT_GAMMA)
     ap.add_argument("--zipf", type=float, default=None)
+    ap.add_argument("--top-k", type=int, default=None,
+                    help="experts per token instead of the config's own (sparsity sweep)")
+    ap.add_argument("--dense-contrast", action="store_true",
+                    help="the rho = 1 layer with the same active parameters per token")
+    ap.add_argument("--grid", default="config", choices=["config", "sparsity"],
+                    help="sweep the config's (B, gamma) grid or the 19 batch sizes x gamma 0/2/4")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep-steps", type=int, default=10)
@@ -303,14 +326,14 @@ def main():
     device = torch.device("cuda", local_rank)
     peaks = load_peaks()
 
-    shape = wl.CONFIGS[args.config]
+    shape = variant_shape(args)
     B, gamma = args.B, args.gamma
     T = B * (gamma + 1)
     w_dev = wl.make_weights(shape, wl.config_seed(args.config), device, zipf_s=args.zipf)
     runner = LayerRunner(shape, w_dev, device)
     max_T = T
     if not args.no_sweep:
-        Bs, gs = wl.GRIDS[args.config]
+        Bs, gs = sweep_grid(args)
         max_T = max(max_T, max(Bs) * (max(gs) + 1))
     runner.prepare(max_T)
     seed = replicas.replica_seed(wl.point_seed(args.config, B, gamma), rank)
@@ -349,8 +372,9 @@ def main():
                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"]}
     # DRAM bytes of one launch from the ncu capture summarised in profiles/ (taken on the
     # default workload; it scales with the activated bytes, so other workloads report null)
-    traffic = NCU_GATE_UP_DRAM_BYTES if (args.config, B, gamma, args.zipf) == (
-        DEFAULT_CONFIG, DEFAULT_B, DEFAULT_GAMMA, None) else None
+    default_point = shape is wl.CONFIGS[args.config] and (args.config, B, gamma, args.zipf) == (
+        DEFAULT_CONFIG, DEFAULT_B, DEFAULT_GAMMA, None)
+    traffic = NCU_GATE_UP_DRAM_BYTES if default_point else None
     roofline.update({"traffic": traffic, "kernel": "ffn_fused_kernel<gate/up + SwiGLU>",
                      "kernel_ms": k_ms, "algorithmic_bytes": gu_bytes,
                      "peak_source": peaks["source"]})
@@ -373,7 +397,7 @@ def main():
     # ---- sweep of the config's (B, gamma) grid ----------------------------------------
     sweep = []
     if not args.no_sweep and rank == 0:
-        Bs, gs = wl.GRIDS[args.config]
+        Bs, gs = sweep_grid(args)
         for Bi in Bs:
             base_ms = None
             for gi in gs:

@@ -77,10 +77,12 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // k chunks the shared expert's down projection is split into inside moe_verify_layer (each
 // chunk is a work unit of its own and writes a partial [T,H] plane that the combine step sums)
 int shared_down_parts(const moe_config_t &c);
-// k chunks of the routed groups' down projection for T tokens (1 above a few tokens)
-constexpr int ROUTED_SPLIT_MAX_TOKENS = 16;
+// k chunks of the routed groups' down projection for T tokens (1 once the pass has enough
+// work items without), and the largest assignment count A' = T' * top_k over T' <= T at which
+// the chunks are still used: y must hold ROUTED_SPLIT_MAX_PARTS planes of A' rows.
 constexpr int ROUTED_SPLIT_MAX_PARTS = 8;
 int routed_down_parts(const moe_config_t &c, int T);
+size_t routed_split_max_rows(const moe_config_t &c, int T);
 
 inline Workspace workspace_layout(const moe_config_t &c, int T)
 {
@@ -111,10 +113,9 @@ inline Workspace workspace_layout(const moe_config_t &c, int T)
     w.x_sorted = take(A * H * 2);
     w.h = take(A * (size_t)c.inter * 2);
     w.h_shared = take((size_t)T * c.shared_inter * 2);
-    // y: [A,H], or for few tokens up to ROUTED_SPLIT_MAX_PARTS partial planes of it
-    const size_t A_small = A < (size_t)ROUTED_SPLIT_MAX_TOKENS * c.top_k
-                               ? A : (size_t)ROUTED_SPLIT_MAX_TOKENS * c.top_k;
-    const size_t y_rows = A > ROUTED_SPLIT_MAX_PARTS * A_small ? A : ROUTED_SPLIT_MAX_PARTS * A_small;
+    // y: [A,H], or while the down pass is short of work items partial planes of it
+    const size_t A_split = ROUTED_SPLIT_MAX_PARTS * routed_split_max_rows(c, T);
+    const size_t y_rows = A > A_split ? A : A_split;
     w.y = take(y_rows * H * 2);
     w.y_shared = take((size_t)T * H * 2 * shared_down_parts(c));
     w.total = off;

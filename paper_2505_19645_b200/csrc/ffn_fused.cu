@@ -1281,17 +1281,25 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
 static int split_chunk(int K, int parts) { return ((K + parts - 1) / parts + 127) / 128 * 128; }
 static int split_parts(int K, int parts) { return (K + split_chunk(K, parts) - 1) / split_chunk(K, parts); }
 
-// k chunks of the routed groups' down projection.  With few tokens the pass has fewer
-// (pair, tile) items than CTAs and one SM cannot pull a tile faster than a fraction of what
-// HBM delivers, so the reduction is cut until about three items per CTA exist; each chunk
-// writes its own plane of y and the combine adds the planes.  Only for T <= 16 (the planes
-// must fit the workspace) and only where the pass deals single items.
+// Expected number of (segment pair, tile) items of the routed down pass; never decreases
+// with T.
+static double routed_down_items(const moe_config_t &c, int T)
+{
+    const double n_act = expected_active_experts(c.n_experts, c.top_k, T);
+    const double rows_per_group = (double)T * c.top_k / n_act;
+    return ceil(n_act) * ceil(ceil(rows_per_group / FF_SEG) / 2.0) * ((c.hidden + 255) / 256);
+}
+
+// k chunks of the routed groups' down projection.  While the pass has fewer than about three
+// (pair, tile) items per CTA -- few tokens, or few experts with long reductions -- some SMs
+// have no weight stream to pull and one SM cannot pull a tile faster than a fraction of what
+// HBM delivers, so the reduction is cut; each chunk writes its own plane of y and the combine
+// adds the planes.  (Fewer than three items per CTA also means the pass deals single items.)
 int routed_down_parts(const moe_config_t &c, int T)
 {
-    if (T > ROUTED_SPLIT_MAX_TOKENS || !use_round_robin(c, T, c.hidden, c.inter, 256, ffn_grid()))
+    if (!use_round_robin(c, T, c.hidden, c.inter, 256, ffn_grid()))
         return 1;
-    const double items = ceil(expected_active_experts(c.n_experts, c.top_k, T)) * ((c.hidden + 255) / 256);
-    int parts = (int)ceil(3.0 * ffn_grid() / items);
+    int parts = (int)ceil(3.0 * ffn_grid() / routed_down_items(c, T));
     const int cap = c.inter / 1024;  // chunks below half a megabyte cost more than they level
     if (parts > cap)
         parts = cap;
@@ -1300,11 +1308,35 @@ int routed_down_parts(const moe_config_t &c, int T)
     return parts < 1 ? 1 : split_parts(c.inter, parts);
 }
 
+size_t routed_split_max_rows(const moe_config_t &c, int T)
+{
+    if (c.inter / 1024 < 2)
+        return 0;
+    // largest T' <= T whose item count still asks for more than one part
+    auto split = [&](int t) { return routed_down_items(c, t) < 3.0 * ffn_grid(); };
+    if (!split(1))
+        return 0;
+    int lo = 1, hi = T;  // split(lo) holds
+    if (split(hi))
+        return (size_t)hi * c.top_k;
+    while (hi - lo > 1) {
+        const int mid = lo + (hi - lo) / 2;
+        if (split(mid))
+            lo = mid;
+        else
+            hi = mid;
+    }
+    return (size_t)lo * c.top_k;
+}
+
 int shared_down_parts(const moe_config_t &c)
 {
-    if (c.shared_inter < 2 * c.inter)
+    // a chunk about as long as a routed expert's reduction, and no longer than 2560 columns
+    int s = c.shared_inter / c.inter;
+    if (s < c.shared_inter / 2560)
+        s = c.shared_inter / 2560;
+    if (s < 2)
         return 1;
-    const int s = c.shared_inter / c.inter;
     return split_parts(c.shared_inter, s > 8 ? 8 : s);
 }
 

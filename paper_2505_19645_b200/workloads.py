@@ -66,6 +66,29 @@ GRIDS = {
 }
 
 
+# Sparsity sweep on one shape (Sec. 4.3 varies the experts per token K of the Qwen2-57B-A14B
+# model, at draft lengths 2 and 4, over these 19 batch sizes).  The paper does not list its
+# six K values; these six span rho = K/E from 1/64 to 1/4 and include the model's own K = 8.
+SPARSITY_BATCHES = [1, 2, 4, 8, 12, 16, 20, 24, 28, 32, 36, 40, 44, 48, 52, 56, 60, 80, 100]
+SPARSITY_GAMMAS = [0, 2, 4]      # gamma = 0 is the denominator T(B, 0) of the cost ratio
+SPARSITY_TOP_KS = [1, 2, 4, 8, 12, 16]
+
+
+def with_top_k(shape: LayerShape, top_k: int) -> LayerShape:
+    """The same layer with K experts per token (a run-time parameter of the routing)."""
+    d = shape.as_dict()
+    d.update(name="%s-k%d" % (shape.name, top_k), top_k=top_k)
+    return LayerShape(**d)
+
+
+def dense_contrast(shape: LayerShape) -> LayerShape:
+    """The rho = 1 limit of Sec. 3.3 with the same active parameters per token: one routed
+    expert of width K*I that every token uses (plus the unchanged shared expert)."""
+    d = shape.as_dict()
+    d.update(name="%s-dense" % shape.name, n_experts=1, top_k=1, inter=shape.top_k * shape.inter)
+    return LayerShape(**d)
+
+
 def config_seed(name: str) -> int:
     """Weight seed of a config: 0 for the tiny config, 1000*index otherwise."""
     return 1000 * CONFIG_ORDER.index(name)

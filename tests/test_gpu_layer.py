@@ -28,6 +28,10 @@ def test_tiny_config_full_parity():
     ("mixtral-like", 512, 8, 2, 1792, 0, 0, 1, 0, 64, 2, None),        # 48 rows per expert
     ("ragged", 160, 6, 3, 224, 96, 0, 1, 0, 11, 6, None),              # row tails everywhere
     ("dense-limit", 128, 4, 4, 256, 0, 0, 1, 0, 5, 1, None),           # k = E
+    # few experts with long reductions: the routed down pass is cut into k chunks
+    ("ksplit-routed", 256, 4, 2, 4096, 0, 0, 1, 0, 10, 3, None),       # four planes of y
+    ("ksplit-odd", 384, 8, 2, 2176, 0, 0, 1, 0, 3, 2, None),           # two chunks, ragged second
+    ("dense-contrast", 256, 1, 1, 3072, 3072, 0, 0, 1, 65, 1, None),   # E = k = 1, 130 rows
 ])
 def test_layer_parity_small_shapes(name, H, E, k, I, Is, score, renorm, sgate, B, gamma, zipf):
     shape = wl.small_shape(name, H, E, k, I, Is, score, renorm, sgate)

@@ -66,6 +66,33 @@ def test_workspace_bytes_and_host_side_validation():
     assert st == 1
 
 
+def test_workspace_bytes_never_shrink_with_the_token_count():
+    """A workspace sized for max_tokens must serve every smaller call, also where the small
+    calls keep several partial planes of the routed output."""
+    from paper_2505_19645_b200 import api
+
+    for name in ("qwen2-57b-a14b", "mixtral-8x7b", "deepseek-v3"):
+        for shape in (wl.CONFIGS[name], wl.dense_contrast(wl.CONFIGS[name]),
+                      wl.with_top_k(wl.CONFIGS[name], 1)):
+            cfg = api.make_config(shape)
+            sizes = [api.moe_workspace_bytes(cfg, t) for t in range(1, 700, 7)]
+            assert all(a <= b for a, b in zip(sizes, sizes[1:])), shape.name
+            A, H = 694 * shape.top_k, shape.hidden
+            assert sizes[-1] >= A * (H + shape.inter) * 2
+
+
+def test_workload_variants_keep_the_active_parameters():
+    base = wl.CONFIGS["qwen2-57b-a14b"]
+    dense = wl.dense_contrast(base)
+    assert (dense.n_experts, dense.top_k) == (1, 1)
+    assert dense.top_k * dense.inter == base.top_k * base.inter
+    assert dense.shared_inter == base.shared_inter and dense.hidden == base.hidden
+    for k in wl.SPARSITY_TOP_KS:
+        v = wl.with_top_k(base, k)
+        assert v.top_k == k and v.n_experts == base.n_experts and v.inter == base.inter
+    assert len(wl.SPARSITY_BATCHES) == 19 and base.top_k in wl.SPARSITY_TOP_KS
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     from paper_2505_19645_b200 import api
 
