@@ -440,7 +440,7 @@ def main():
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic (seeded)",
             "config": {"workload": workload_name(args), "config": args.config, "B": B,
-                       "gamma": gamma, "tokens": T, "zipf": args.zipf,
+                       "gamma": gamma, "tokens": T, "zipf": args.zipf, "shape": shape.as_dict(),
                        "l2": "512 MiB buffer written between timed iterations",
                        "parallelism": "replicas only"},
             "roofline": roofline, "layer_roofline": layer_roof, "cpu_baseline": cpu,
