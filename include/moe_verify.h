@@ -191,7 +191,9 @@ moe_status_t moe_check(void *ws, void *stream);
  * time to weight loading, which the benchmark verifies per kernel).  Every following
  * moe_verify_layer call of this thread records start_event before and stop_event after the
  * kernel of the given stage on the call's stream.  Events are cudaEvent_t passed as void*,
- * created and owned by the caller; stage < 0 switches the recording off. */
+ * created and owned by the caller; stage < 0 switches the recording off.  A stage whose work
+ * another stage's kernel does for the call's size (small batches: top-k and gather inside the
+ * grouping kernel) records nothing. */
 typedef enum {
     MOE_STAGE_ROUTER_LOGITS = 0,
     MOE_STAGE_ROUTE_TOPK = 1,

@@ -141,7 +141,8 @@ PlanView plan_view(char *ws, const Workspace &L)
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
                      const int32_t *offsets, const int32_t *perm, __nv_bfloat16 *y,
                      __nv_bfloat16 *shared_y, char *ws, const Workspace &L, cudaStream_t s,
-                     int &launches, bool plan_ready, int shared_parts, int routed_parts)
+                     int &launches, bool plan_ready, int shared_parts, int routed_parts,
+                     bool gathered)
 {
     const bool with_shared = shared_y != nullptr && c.shared_inter > 0;
     const PlanView plan = plan_view(ws, L);
@@ -151,7 +152,8 @@ moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_b
     __nv_bfloat16 *xs = reinterpret_cast<__nv_bfloat16 *>(ws + L.x_sorted);
     if (!plan_ready)
         MOE_STAGE(MOE_STAGE_PLAN, launch_plan(c, T, offsets, status, plan, s));
-    MOE_STAGE(MOE_STAGE_GATHER, launch_gather_rows(c, x, perm, T, xs, s));
+    if (!gathered)
+        MOE_STAGE(MOE_STAGE_GATHER, launch_gather_rows(c, x, perm, T, xs, s));
     MOE_STAGE(MOE_STAGE_GATE_UP,
               launch_ffn_gateup(c, w, x, xs, T, plan, with_shared, h, hs, status, s));
     MOE_STAGE(MOE_STAGE_DOWN,
@@ -328,16 +330,26 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
     MOE_STAGE(MOE_STAGE_ROUTER_LOGITS,
               launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s,
                                    plan_view(base, L).done_shared, max_shared_segments(T)));
-    MOE_STAGE(MOE_STAGE_ROUTE_TOPK, launch_route_topk(*cfg, logits, T, topk_idx, topk_w, s));
-    // the grouping kernel also writes the FFN segment plan (one launch fewer)
+    // the grouping kernel also writes the FFN segment plan (one launch fewer); for a small
+    // batch it selects the experts and gathers the token rows as well (three fewer)
     const PlanView plan = plan_view(base, L);
-    MOE_STAGE(MOE_STAGE_PERMUTE,
-              launch_permute(*cfg, topk_idx, T, counts, offsets, perm, inv_perm, active, n_active, s,
-                             &plan, reinterpret_cast<int32_t *>(base + L.status)));
+    int32_t *status = reinterpret_cast<int32_t *>(base + L.status);
+    const bool small = route_group_small_applies(*cfg, T);
+    if (small) {
+        MOE_STAGE(MOE_STAGE_PERMUTE,
+                  launch_route_group_small(*cfg, logits, xb, T, topk_idx, topk_w, counts, offsets,
+                                           perm, inv_perm, active, n_active, status, plan,
+                                           reinterpret_cast<__nv_bfloat16 *>(base + L.x_sorted), s));
+    } else {
+        MOE_STAGE(MOE_STAGE_ROUTE_TOPK, launch_route_topk(*cfg, logits, T, topk_idx, topk_w, s));
+        MOE_STAGE(MOE_STAGE_PERMUTE,
+                  launch_permute(*cfg, topk_idx, T, counts, offsets, perm, inv_perm, active,
+                                 n_active, s, &plan, status));
+    }
     const int shared_parts = has_shared ? shared_down_parts(*cfg) : 1;
     const int routed_parts = routed_down_parts(*cfg, T);
     st = run_ffn(*cfg, *w, xb, T, offsets, perm, y, ys, base, L, s, launches, true, shared_parts,
-                 routed_parts);
+                 routed_parts, small);
     if (st != MOE_OK)
         return st;
     MOE_STAGE(MOE_STAGE_COMBINE,

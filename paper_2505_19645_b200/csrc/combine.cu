@@ -7,6 +7,7 @@
 namespace moe {
 
 constexpr int CB_THREADS = 256;
+constexpr int MOE_MAX_SHARED_PARTS = 8;  // k chunks of the shared expert's down pass, at most
 
 __global__ void __launch_bounds__(CB_THREADS)
 combine_kernel(const __nv_bfloat16 *__restrict__ y, int routed_parts,
@@ -60,17 +61,25 @@ combine_kernel(const __nv_bfloat16 *__restrict__ y, int routed_parts,
             }
         }
         if (shared_y) {
-            for (int part = 0; part < shared_parts; ++part) {
-                const uint4 sv = *reinterpret_cast<const uint4 *>(
-                    shared_y + ((size_t)part * T + t) * H + h);
-                acc[0] = fmaf(s, bf16_lo(sv.x), acc[0]);
-                acc[1] = fmaf(s, bf16_hi(sv.x), acc[1]);
-                acc[2] = fmaf(s, bf16_lo(sv.y), acc[2]);
-                acc[3] = fmaf(s, bf16_hi(sv.y), acc[3]);
-                acc[4] = fmaf(s, bf16_lo(sv.z), acc[4]);
-                acc[5] = fmaf(s, bf16_hi(sv.z), acc[5]);
-                acc[6] = fmaf(s, bf16_lo(sv.w), acc[6]);
-                acc[7] = fmaf(s, bf16_hi(sv.w), acc[7]);
+            // all planes requested before the first one is used
+            uint4 sv[MOE_MAX_SHARED_PARTS];
+#pragma unroll
+            for (int part = 0; part < MOE_MAX_SHARED_PARTS; ++part)
+                if (part < shared_parts)
+                    sv[part] = *reinterpret_cast<const uint4 *>(
+                        shared_y + ((size_t)part * T + t) * H + h);
+#pragma unroll
+            for (int part = 0; part < MOE_MAX_SHARED_PARTS; ++part) {
+                if (part < shared_parts) {
+                    acc[0] = fmaf(s, bf16_lo(sv[part].x), acc[0]);
+                    acc[1] = fmaf(s, bf16_hi(sv[part].x), acc[1]);
+                    acc[2] = fmaf(s, bf16_lo(sv[part].y), acc[2]);
+                    acc[3] = fmaf(s, bf16_hi(sv[part].y), acc[3]);
+                    acc[4] = fmaf(s, bf16_lo(sv[part].z), acc[4]);
+                    acc[5] = fmaf(s, bf16_hi(sv[part].z), acc[5]);
+                    acc[6] = fmaf(s, bf16_lo(sv[part].w), acc[6]);
+                    acc[7] = fmaf(s, bf16_hi(sv[part].w), acc[7]);
+                }
             }
         }
         uint4 o;
@@ -92,6 +101,8 @@ cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, int ro
                            const __nv_bfloat16 *shared_y, int shared_parts,
                            const float *shared_scale, int T, __nv_bfloat16 *out, cudaStream_t s)
 {
+    if (shared_parts > MOE_MAX_SHARED_PARTS)
+        return cudaErrorInvalidValue;
     const size_t total = (size_t)T * (c.hidden >> 3);
     size_t blocks = (total + CB_THREADS - 1) / CB_THREADS;
     const size_t cap = (size_t)sm_count() * 8;

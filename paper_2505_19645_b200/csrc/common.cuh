@@ -155,6 +155,15 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
                             __nv_bfloat16 *y, __nv_bfloat16 *y_shared, int shared_parts,
                             int routed_parts,
                             int32_t *status, cudaStream_t s);
+// top-k, grouping, plan and gather of a small batch in one launch (replaces
+// launch_route_topk + launch_permute + launch_gather_rows where it applies)
+bool route_group_small_applies(const moe_config_t &c, int T);
+cudaError_t launch_route_group_small(const moe_config_t &c, const float *logits,
+                                     const __nv_bfloat16 *x, int T, int32_t *topk_idx, float *topk_w,
+                                     int32_t *counts, int32_t *offsets, int32_t *perm,
+                                     int32_t *inv_perm, int32_t *active, int32_t *n_active,
+                                     int32_t *status, PlanView plan, __nv_bfloat16 *x_sorted,
+                                     cudaStream_t s);
 // token rows in sorted order (the token operand of the routed gate/up tiles)
 cudaError_t launch_gather_rows(const moe_config_t &c, const __nv_bfloat16 *x, const int32_t *perm,
                                int T, __nv_bfloat16 *x_sorted, cudaStream_t s);
@@ -180,7 +189,7 @@ moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_b
                      const int32_t *offsets, const int32_t *perm, __nv_bfloat16 *y,
                      __nv_bfloat16 *shared_y, char *ws, const Workspace &L, cudaStream_t s,
                      int &launches, bool plan_ready = false, int shared_parts = 1,
-                     int routed_parts = 1);
+                     int routed_parts = 1, bool gathered = false);
 
 // ---------------------------------------------------------------------------------------
 // Device helpers.

@@ -1063,13 +1063,27 @@ gather_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__restric
     griddep_wait();
     const int vec_per_row = H >> 3;
     const size_t total = (size_t)A * vec_per_row;
-    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total;
-         i += (size_t)gridDim.x * blockDim.x) {
-        const int r = (int)(i / vec_per_row);
-        const int v = (int)(i - (size_t)r * vec_per_row);
-        const int t = perm[r] / top_k;
-        reinterpret_cast<uint4 *>(x_sorted + (size_t)r * H)[v] =
-            reinterpret_cast<const uint4 *>(x + (size_t)t * H)[v];
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    // four independent row pieces per thread and pass: few CTAs (they must leave room for
+    // the FFN CTAs that start beside them) still keep enough loads in flight
+    for (size_t i0 = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i0 < total; i0 += 4 * stride) {
+        int r[4], v[4], t[4];
+        uint4 d[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const size_t i = i0 + u * stride;
+            r[u] = i < total ? (int)(i / vec_per_row) : -1;
+            v[u] = i < total ? (int)(i - (size_t)r[u] * vec_per_row) : 0;
+            t[u] = r[u] >= 0 ? perm[r[u]] / top_k : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (r[u] >= 0)
+                d[u] = reinterpret_cast<const uint4 *>(x + (size_t)t[u] * H)[v[u]];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (r[u] >= 0)
+                reinterpret_cast<uint4 *>(x_sorted + (size_t)r[u] * H)[v[u]] = d[u];
     }
 }
 
@@ -1079,7 +1093,7 @@ cudaError_t launch_gather_rows(const moe_config_t &c, const __nv_bfloat16 *x, co
     const int A = T * c.top_k;
     const size_t total = (size_t)A * (c.hidden >> 3);
     size_t blocks = (total + 255) / 256;
-    const size_t cap = (size_t)sm_count() * 8;
+    const size_t cap = (size_t)sm_count() * 2;
     if (blocks > cap)
         blocks = cap;
     return launch_pdl(gather_rows_kernel, dim3((unsigned)blocks), dim3(256), 0, s, x, perm, A,

@@ -1,10 +1,12 @@
 // Token-to-expert grouping: histogram, exclusive scan, stable placement, active-expert list,
 // and the segment plan the FFN kernels iterate over.
-#include "common.cuh"
+#include "route_topk.cuh"
 
 namespace moe {
 
 constexpr int PERM_THREADS = 1024;  // assignments per CTA, one per thread
+constexpr int ROUTE_SMALL_TOKENS = 32;   // one warp per token in a CTA of PERM_THREADS
+constexpr int ROUTE_SMALL_ASSIGN = 512;  // = ROUTE_SMALL_TOKENS * MOE_MAX_TOPK
 
 // Exclusive scan of vals[0..n) (n <= MOE_MAX_EXPERTS <= blockDim.x) in shared memory;
 // returns the total in *total.  All threads of the block must call it.  Warp shuffles inside
@@ -95,6 +97,36 @@ __device__ void build_plan(const int *cnt_sh, const int *off_sh, int *scan, int 
     }
 }
 
+// counts / offsets / active / n_active from the histogram and its exclusive scan (shared
+// memory, `total` = number of assignments) and, if asked for, the FFN segment plan.  All
+// threads of the block must call it; flag/tmp are shared scratch of MOE_MAX_EXPERTS ints.
+__device__ void write_tables(int *hist, int *offs, int *flag, int *tmp, int *total, int E,
+                             int32_t *counts, int32_t *offsets, int32_t *active, int32_t *n_active,
+                             int32_t *status, PlanView plan)
+{
+    const int tid = threadIdx.x;
+    __syncthreads();
+    if (tid < E) {
+        counts[tid] = hist[tid];
+        offsets[tid] = offs[tid];
+    }
+    if (tid == 0)
+        offsets[E] = *total;
+    if (tid < MOE_MAX_EXPERTS)
+        flag[tid] = (tid < E && hist[tid] > 0) ? 1 : 0;
+    __syncthreads();
+    const int my_flag = tid < E ? flag[tid] : 0;
+    block_exclusive_scan(flag, tmp, E, total);
+    if (tid < E && my_flag)
+        active[flag[tid]] = tid;
+    if (tid < E && tid >= *total)
+        active[tid] = -1;
+    if (tid == 0)
+        n_active[0] = *total;
+    if (plan.header != nullptr)
+        build_plan(hist, offs, flag, tmp, total, E, status, plan);
+}
+
 // Adds one to hist[e] for every lane with a valid e.  With few experts a plain per-lane
 // atomic would serialise the block on a handful of counters, so the lanes of a warp that hold
 // the same expert are combined first (one atomic per distinct expert); with many experts the
@@ -176,29 +208,8 @@ permute_kernel(const int32_t *__restrict__ topk_idx, int A, int E, int32_t *__re
         inv_perm[my_a] = pos;
     }
 
-    if (tables_cta) {
-        int *flag = before;  // this CTA counted no earlier chunk: the table is free (all zero)
-        __syncthreads();
-        if (tid < E) {
-            counts[tid] = hist[tid];
-            offsets[tid] = offs[tid];
-        }
-        if (tid == 0)
-            offsets[E] = total;
-        if (tid < MOE_MAX_EXPERTS)
-            flag[tid] = (tid < E && hist[tid] > 0) ? 1 : 0;
-        __syncthreads();
-        const int my_flag = tid < E ? flag[tid] : 0;
-        block_exclusive_scan(flag, tmp, E, &total);
-        if (tid < E && my_flag)
-            active[flag[tid]] = tid;
-        if (tid < E && tid >= total)
-            active[tid] = -1;
-        if (tid == 0)
-            n_active[0] = total;
-        if (plan.header != nullptr)
-            build_plan(hist, offs, flag, tmp, &total, E, status, plan);
-    }
+    if (tables_cta)  // this CTA counted no earlier chunk: `before` is free (all zero)
+        write_tables(hist, offs, before, tmp, &total, E, counts, offsets, active, n_active, status, plan);
 }
 
 cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int32_t *counts,
@@ -212,6 +223,138 @@ cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int
         pv = *plan;
     return launch_pdl(permute_kernel, dim3(blocks), dim3(PERM_THREADS), 0, s, idx, A, c.n_experts,
                       counts, offsets, perm, inv_perm, active, n_active, status, pv);
+}
+
+// Routing of a small batch in one launch: top-k, grouping, segment plan and the gather of
+// the token rows into sorted order, for T <= ROUTE_SMALL_TOKENS tokens and at most
+// ROUTE_SMALL_ASSIGN assignments.  Every CTA repeats the (tiny) top-k and counting sort for
+// itself, so no CTA waits for another: CTA 0 writes topk_idx / topk_w / perm / inv_perm, CTA 1
+// the tables and the plan, and the others copy the rows x[perm[r] / k] -> x_sorted[r], row r
+// on CTA 2 + r mod (gridDim.x - 2).  Results are those of route_topk_kernel, permute_kernel
+// and gather_rows_kernel run one after the other, with two launch boundaries fewer on the
+// path from the logits to the first routed tile.
+template <int VPL>
+__global__ void __launch_bounds__(PERM_THREADS)
+route_group_small_kernel(const float *__restrict__ logits, const __nv_bfloat16 *__restrict__ x,
+                         int T, int H, int E, int k, int score_fn, int renormalize,
+                         float routed_scale, int32_t *__restrict__ topk_idx,
+                         float *__restrict__ topk_w, int32_t *__restrict__ counts,
+                         int32_t *__restrict__ offsets, int32_t *__restrict__ perm,
+                         int32_t *__restrict__ inv_perm, int32_t *__restrict__ active,
+                         int32_t *__restrict__ n_active, int32_t *__restrict__ status,
+                         PlanView plan, __nv_bfloat16 *__restrict__ x_sorted)
+{
+    __shared__ int hist[MOE_MAX_EXPERTS];
+    __shared__ int offs[MOE_MAX_EXPERTS];
+    __shared__ int tmp[MOE_MAX_EXPERTS];
+    __shared__ int flag[MOE_MAX_EXPERTS];
+    __shared__ uint16_t wcount[ROUTE_SMALL_ASSIGN / 32][MOE_MAX_EXPERTS];
+    __shared__ int expert_of[ROUTE_SMALL_ASSIGN];  // by assignment t * k + j
+    __shared__ int token_of[ROUTE_SMALL_ASSIGN];   // by sorted row
+    __shared__ int total;
+    griddep_launch();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int A = T * k;
+    if (tid < MOE_MAX_EXPERTS)
+        hist[tid] = 0;
+    for (int i = tid; i < (ROUTE_SMALL_ASSIGN / 32) * MOE_MAX_EXPERTS / 2; i += PERM_THREADS)
+        reinterpret_cast<uint32_t *>(&wcount[0][0])[i] = 0u;
+    griddep_wait();  // the logits come from the preceding kernel
+
+    // top-k: warp w selects for token w
+    if (warp < T) {
+        int sel_i;
+        float sel_w;
+        warp_route_topk<VPL>(logits + (size_t)warp * E, E, k, score_fn, renormalize, routed_scale,
+                             lane, sel_i, sel_w);
+        if (lane < k) {
+            expert_of[warp * k + lane] = sel_i;
+            if (blockIdx.x == 0) {
+                topk_idx[warp * k + lane] = sel_i;
+                topk_w[warp * k + lane] = sel_w;
+            }
+        }
+    }
+    __syncthreads();
+
+    // counting sort, one assignment per thread (threads beyond A idle along)
+    const bool few = E <= 32;
+    const int my_e = tid < A ? expert_of[tid] : -1;
+    const bool my_valid = my_e >= 0 && my_e < E;
+    warp_histogram_add(hist, my_e, my_valid, few);
+    const uint32_t peers = __match_any_sync(0xffffffffu, my_valid ? my_e : -1);
+    const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+    if (my_valid && lane == __ffs(peers) - 1)
+        wcount[warp][my_e] = (uint16_t)__popc(peers);
+    __syncthreads();
+    if (tid < MOE_MAX_EXPERTS)
+        offs[tid] = tid < E ? hist[tid] : 0;
+    __syncthreads();
+    block_exclusive_scan(offs, tmp, E, &total);
+    int pos = 0;
+    if (my_valid) {
+        pos = offs[my_e] + rank_in_warp;
+        for (int w = 0; w < warp; ++w)
+            pos += wcount[w][my_e];
+    }
+
+    if (blockIdx.x == 0) {
+        if (my_valid) {
+            perm[pos] = tid;
+            inv_perm[tid] = pos;
+        }
+    } else if (blockIdx.x == 1) {
+        write_tables(hist, offs, flag, tmp, &total, E, counts, offsets, active, n_active, status, plan);
+    } else {
+        if (my_valid)
+            token_of[pos] = tid / k;
+        __syncthreads();
+        const int vec_per_row = H >> 3;
+        const int n_copy = gridDim.x - 2;
+        for (int r = blockIdx.x - 2; r < A; r += n_copy) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)token_of[r] * H);
+            uint4 *dst = reinterpret_cast<uint4 *>(x_sorted + (size_t)r * H);
+            for (int v = tid; v < vec_per_row; v += PERM_THREADS)
+                dst[v] = src[v];
+        }
+    }
+}
+
+bool route_group_small_applies(const moe_config_t &c, int T)
+{
+    return T <= ROUTE_SMALL_TOKENS && T * c.top_k <= ROUTE_SMALL_ASSIGN;
+}
+
+cudaError_t launch_route_group_small(const moe_config_t &c, const float *logits,
+                                     const __nv_bfloat16 *x, int T, int32_t *topk_idx, float *topk_w,
+                                     int32_t *counts, int32_t *offsets, int32_t *perm,
+                                     int32_t *inv_perm, int32_t *active, int32_t *n_active,
+                                     int32_t *status, PlanView plan, __nv_bfloat16 *x_sorted,
+                                     cudaStream_t s)
+{
+    if (!route_group_small_applies(c, T))
+        return cudaErrorInvalidValue;
+    const int A = T * c.top_k, E = c.n_experts;
+    // copy CTAs: one per sorted row up to 64 (a CTA moves a row of H values in one or two steps)
+    const int blocks = 2 + (A < 64 ? A : 64);
+#define MOE_RG_LAUNCH(V)                                                                         \
+    err = launch_pdl(route_group_small_kernel<V>, dim3(blocks), dim3(PERM_THREADS), 0, s, logits, \
+                     x, T, c.hidden, E, c.top_k, c.score_fn, c.renormalize, c.routed_scale,       \
+                     topk_idx, topk_w, counts, offsets, perm, inv_perm, active, n_active, status, \
+                     plan, x_sorted)
+    cudaError_t err = cudaSuccess;
+    if (E <= 32)
+        MOE_RG_LAUNCH(1);
+    else if (E <= 64)
+        MOE_RG_LAUNCH(2);
+    else if (E <= 128)
+        MOE_RG_LAUNCH(4);
+    else if (E <= 256)
+        MOE_RG_LAUNCH(8);
+    else
+        MOE_RG_LAUNCH(16);
+#undef MOE_RG_LAUNCH
+    return err;
 }
 
 // Stand-alone plan (moe_grouped_swiglu gets its offsets from the caller).

@@ -1,17 +1,9 @@
-// Router: fp32 logits (x . w_router^T + bias), the shared expert's scalar gate, and the
-// warp-per-token top-k selection with softmax / sigmoid gate weights.
-#include <float.h>
-
-#include "common.cuh"
+// Top-k routing kernel: one warp per token selects the k experts and their softmax / sigmoid
+// gate weights from the fp32 logits.
+#include "route_topk.cuh"
 
 namespace moe {
 
-
-// ---------------------------------------------------------------------------------------
-// Top-k.  One warp per token; lane l holds logits l, l+32, ...  Selection runs k rounds of
-// a warp arg-max on the raw fp32 logits (ties: lower expert index), so it is exact and
-// independent of the score function.  Scores use expf.
-// ---------------------------------------------------------------------------------------
 template <int VPL>
 __global__ void __launch_bounds__(128)
 route_topk_kernel(const float *__restrict__ logits, int T, int E, int k, int score_fn,
@@ -24,78 +16,13 @@ route_topk_kernel(const float *__restrict__ logits, int T, int E, int k, int sco
     const int t = (int)((blockIdx.x * (size_t)blockDim.x + threadIdx.x) >> 5);
     if (t >= T)
         return;
-    const float *z = logits + (size_t)t * E;
-    float v[VPL];
-    float vmax = -FLT_MAX;
-#pragma unroll
-    for (int i = 0; i < VPL; ++i) {
-        const int e = lane + 32 * i;
-        v[i] = e < E ? z[e] : -FLT_MAX;
-        vmax = fmaxf(vmax, v[i]);
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1)
-        vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, off));
-    float denom = 1.f;
-    if (score_fn == MOE_SCORE_SOFTMAX) {
-        float sum = 0.f;
-#pragma unroll
-        for (int i = 0; i < VPL; ++i)
-            if (lane + 32 * i < E)
-                sum += expf(v[i] - vmax);
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1)
-            sum += __shfl_xor_sync(0xffffffffu, sum, off);
-        denom = sum;
-    }
-
-    uint32_t taken = 0;
-    float sel_v = 0.f;
-    int sel_i = 0;
-    for (int j = 0; j < k; ++j) {
-        float bv = -FLT_MAX;
-        int bi = 0x7fffffff;
-#pragma unroll
-        for (int i = 0; i < VPL; ++i) {
-            const int e = lane + 32 * i;
-            if (e < E && !((taken >> i) & 1u) && (bi == 0x7fffffff || v[i] > bv)) {
-                bv = v[i];
-                bi = e;
-            }
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-            if (oi != 0x7fffffff && (bi == 0x7fffffff || ov > bv || (ov == bv && oi < bi))) {
-                bv = ov;
-                bi = oi;
-            }
-        }
-        if (bi != 0x7fffffff && (bi & 31) == lane)
-            taken |= 1u << (bi >> 5);
-        if (lane == j) {
-            sel_v = bv;
-            sel_i = bi;
-        }
-    }
-    float p = 0.f;
-    if (lane < k) {
-        if (score_fn == MOE_SCORE_SOFTMAX)
-            p = expf(sel_v - vmax) / denom;
-        else
-            p = 1.0f / (1.0f + expf(-sel_v));
-    }
-    if (renormalize) {
-        float s = p;
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1)
-            s += __shfl_xor_sync(0xffffffffu, s, off);
-        p = p / s;
-    }
+    int sel_i;
+    float sel_w;
+    warp_route_topk<VPL>(logits + (size_t)t * E, E, k, score_fn, renormalize, routed_scale, lane,
+                         sel_i, sel_w);
     if (lane < k) {
         topk_idx[(size_t)t * k + lane] = sel_i;
-        topk_w[(size_t)t * k + lane] = p * routed_scale;
+        topk_w[(size_t)t * k + lane] = sel_w;
     }
 }
 
