@@ -916,7 +916,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 for (int k0 = it.k0; ok && k0 < K; k0 += 64 * kb) {
                     const int nbox = min(kb, (K - k0 + 63) >> 6);
                     // the weight slot is multiplied with one or two segments' token entries
-                    uint32_t xbase[2];
+                    uint32_t xbase[2], xpar[2];
                     int xe[2], pieces[2];
                     for (int sub = 0; sub < nsub; ++sub) {
                         pieces[sub] = pieces16(sub ? it2.n : it.n);
@@ -924,18 +924,22 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                         int pad;
                         const int at = ring.place(pieces[sub] * kb, pad);
                         xe[sub] = j % FF_X_ENTRIES;
+                        xpar[sub] = (uint32_t)(j / FF_X_ENTRIES) & 1u;
                         xbase[sub] = ring_x + (uint32_t)at * FF_X_UNIT;
-                        if (!mbar_wait(x_full(xe[sub]), (uint32_t)(j / FF_X_ENTRIES) & 1u, abortp,
-                                       args.status))
-                            ok = false;
                     }
-                    if (!ok || !mbar_wait(w_full(sw), pw, abortp, args.status)) {
+                    if (!mbar_wait(w_full(sw), pw, abortp, args.status)) {
                         ok = false;
                         break;
                     }
-                    tc_fence_after();
                     const uint32_t wbase = ring_w + sw * args.w_slot_bytes;
                     for (int sub = 0; sub < nsub; ++sub) {
+                        // the second segment's rows may still be landing while the first
+                        // segment's instructions run
+                        if (!mbar_wait(x_full(xe[sub]), xpar[sub], abortp, args.status)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
                         if (!acc_ready[sub]) {
                             if (!mbar_wait(acc_empty(buf[sub]), acc_par[sub], abortp, args.status)) {
                                 ok = false;
