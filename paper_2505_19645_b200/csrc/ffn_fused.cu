@@ -799,8 +799,8 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             int seen[2] = {-1, -1};  // (group, segment) keys last found complete
             const uint64_t pol_keep = l2_policy_evict_last();
             int released = 0;          // entries known to have been consumed
-            int v_cur = 0, v_rel = 0;  // virtual unit positions: issued up to / released up to
-            int v_end_of[FF_X_ENTRIES];
+            int v_cur = 0, v_rel = 0;  // virtual unit positions: issued up to / free up to
+            int v_start_of[FF_X_ENTRIES];  // where each entry's rows begin (after its padding)
             bool ok = true;
             Item it;
             while (ok && walk.next(it)) {
@@ -836,9 +836,10 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                         const int j = ring.count;
                         int pad;
                         const int at = ring.place(m, pad);
-                        const int v_end = v_cur + pad + m;
-                        // the entry's units (and its barrier pair) must have been released
-                        // (with nothing outstanding the whole ring is free, padding included)
+                        const int v_start = v_cur + pad, v_end = v_start + m;
+                        // the entry's units (and its barrier pair) must have been released:
+                        // everything before the oldest entry still in use is free, the
+                        // padding in front of it included
                         while (released < j &&
                                (j - released >= FF_X_ENTRIES || v_end - v_rel > args.x_units)) {
                             const int r = released % FF_X_ENTRIES;
@@ -847,13 +848,13 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                                 ok = false;
                                 break;
                             }
-                            v_rel = v_end_of[r];
                             ++released;
+                            v_rel = released < j ? v_start_of[released % FF_X_ENTRIES] : v_start;
                         }
                         if (!ok)
                             break;
                         const int e = j % FF_X_ENTRIES;
-                        v_end_of[e] = v_end;
+                        v_start_of[e] = v_start;
                         v_cur = v_end;
                         const uint32_t base = ring_x + (uint32_t)at * FF_X_UNIT;
                         mbar_expect_tx(x_full(e), (uint32_t)(nbox * pieces) * FF_X_UNIT);
@@ -1197,6 +1198,12 @@ static void ffn_geometry(int T, FfnArgs &a)
     int x_ring_bytes = T > 64 ? 96 * 1024 : 32 * 1024;
     if (exr)
         x_ring_bytes = atoi(exr) * 1024;
+    // entries never wrap, so two entries that must be resident together (a pair of segments:
+    // 32 KB + up to 32 KB) need a ring of three of them wherever the first may sit
+    if (T > 64 && x_ring_bytes < 96 * 1024)
+        x_ring_bytes = 96 * 1024;
+    if (x_ring_bytes < 32 * 1024)
+        x_ring_bytes = 32 * 1024;
     a.x_units = x_ring_bytes / FF_X_UNIT;
     const int avail = FF_SMEM_LIMIT - 1024 - 512;  // alignment slack, static shared memory
     int ns = (avail - x_ring_bytes) / a.w_slot_bytes;
