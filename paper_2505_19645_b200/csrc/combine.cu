@@ -9,78 +9,84 @@ namespace moe {
 constexpr int CB_THREADS = 256;
 constexpr int MOE_MAX_SHARED_PARTS = 8;  // k chunks of the shared expert's down pass, at most
 
-__global__ void __launch_bounds__(CB_THREADS)
+__device__ __forceinline__ void accumulate8(float (&acc)[8], float w, const uint4 &v)
+{
+    acc[0] = fmaf(w, bf16_lo(v.x), acc[0]);
+    acc[1] = fmaf(w, bf16_hi(v.x), acc[1]);
+    acc[2] = fmaf(w, bf16_lo(v.y), acc[2]);
+    acc[3] = fmaf(w, bf16_hi(v.y), acc[3]);
+    acc[4] = fmaf(w, bf16_lo(v.z), acc[4]);
+    acc[5] = fmaf(w, bf16_hi(v.z), acc[5]);
+    acc[6] = fmaf(w, bf16_lo(v.w), acc[6]);
+    acc[7] = fmaf(w, bf16_hi(v.w), acc[7]);
+}
+
+// KP: top_k rounded up to 2, 4, 8 or 16 -- the arrays of row pieces in flight are sized by it,
+// so that a top-2 or top-4 layer keeps its registers (and its occupancy).
+template <int KP>
+__global__ void __launch_bounds__(CB_THREADS, KP <= 2 ? 4 : (KP <= 4 ? 3 : (KP <= 8 ? 2 : 1)))
 combine_kernel(const __nv_bfloat16 *__restrict__ y, int routed_parts,
-               const int32_t *__restrict__ inv_perm,
-               const float *__restrict__ topk_w, const __nv_bfloat16 *__restrict__ shared_y,
-               int shared_parts, const float *__restrict__ shared_scale, int T, int H, int k,
+               const int32_t *__restrict__ inv_perm, const float *__restrict__ topk_w,
+               const __nv_bfloat16 *__restrict__ shared_y, int shared_parts,
+               const float *__restrict__ shared_scale, int T, int H, int k,
                __nv_bfloat16 *__restrict__ out)
 {
     griddep_launch();
     griddep_wait();  // y and shared_y come from the preceding kernel
     const int vec_per_row = H >> 3;
     const size_t total = (size_t)T * vec_per_row;
+    const size_t plane = (size_t)T * k * H;
     for (size_t i = blockIdx.x * (size_t)CB_THREADS + threadIdx.x; i < total;
          i += (size_t)gridDim.x * CB_THREADS) {
         const int t = (int)(i / vec_per_row);
         const int h = (int)(i - (size_t)t * vec_per_row) << 3;
-        // the k rows of this token: positions and weights first, then all row pieces, so that
-        // the loads of one level are in flight together
-        int rows[MOE_MAX_TOPK];
-        float wts[MOE_MAX_TOPK];
+        // the k rows of this token: positions and weights first, then the row pieces of a
+        // plane, so that the loads of one level are in flight together
+        int rows[KP];
+        float wts[KP];
 #pragma unroll
-        for (int j = 0; j < MOE_MAX_TOPK; ++j) {
+        for (int j = 0; j < KP; ++j) {
             rows[j] = j < k ? inv_perm[(size_t)t * k + j] : 0;
             wts[j] = j < k ? topk_w[(size_t)t * k + j] : 0.f;
         }
         const float s = shared_y && shared_scale ? shared_scale[t] : 1.0f;
+        // the shared expert's planes, four at a time, requested before the routed rows are used
+        uint4 sv[4];
+        const int sp0 = shared_y ? (shared_parts < 4 ? shared_parts : 4) : 0;
+#pragma unroll
+        for (int p = 0; p < 4; ++p)
+            if (p < sp0)
+                sv[p] = *reinterpret_cast<const uint4 *>(shared_y + ((size_t)p * T + t) * H + h);
         float acc[8];
 #pragma unroll
         for (int q = 0; q < 8; ++q)
             acc[q] = 0.f;
         for (int part = 0; part < routed_parts; ++part) {
-            const __nv_bfloat16 *yp = y + (size_t)part * T * k * H;
-            uint4 v[MOE_MAX_TOPK];
+            const __nv_bfloat16 *yp = y + (size_t)part * plane;
+            uint4 v[KP];
 #pragma unroll
-            for (int j = 0; j < MOE_MAX_TOPK; ++j)
+            for (int j = 0; j < KP; ++j)
                 if (j < k)
                     v[j] = *reinterpret_cast<const uint4 *>(yp + (size_t)rows[j] * H + h);
 #pragma unroll
-            for (int j = 0; j < MOE_MAX_TOPK; ++j) {
-                if (j < k) {
-                    const float w = wts[j];
-                    acc[0] = fmaf(w, bf16_lo(v[j].x), acc[0]);
-                    acc[1] = fmaf(w, bf16_hi(v[j].x), acc[1]);
-                    acc[2] = fmaf(w, bf16_lo(v[j].y), acc[2]);
-                    acc[3] = fmaf(w, bf16_hi(v[j].y), acc[3]);
-                    acc[4] = fmaf(w, bf16_lo(v[j].z), acc[4]);
-                    acc[5] = fmaf(w, bf16_hi(v[j].z), acc[5]);
-                    acc[6] = fmaf(w, bf16_lo(v[j].w), acc[6]);
-                    acc[7] = fmaf(w, bf16_hi(v[j].w), acc[7]);
-                }
-            }
+            for (int j = 0; j < KP; ++j)
+                if (j < k)
+                    accumulate8(acc, wts[j], v[j]);
         }
-        if (shared_y) {
-            // all planes requested before the first one is used
-            uint4 sv[MOE_MAX_SHARED_PARTS];
 #pragma unroll
-            for (int part = 0; part < MOE_MAX_SHARED_PARTS; ++part)
-                if (part < shared_parts)
-                    sv[part] = *reinterpret_cast<const uint4 *>(
-                        shared_y + ((size_t)part * T + t) * H + h);
+        for (int p = 0; p < 4; ++p)
+            if (p < sp0)
+                accumulate8(acc, s, sv[p]);
+        if (shared_y && shared_parts > 4) {
 #pragma unroll
-            for (int part = 0; part < MOE_MAX_SHARED_PARTS; ++part) {
-                if (part < shared_parts) {
-                    acc[0] = fmaf(s, bf16_lo(sv[part].x), acc[0]);
-                    acc[1] = fmaf(s, bf16_hi(sv[part].x), acc[1]);
-                    acc[2] = fmaf(s, bf16_lo(sv[part].y), acc[2]);
-                    acc[3] = fmaf(s, bf16_hi(sv[part].y), acc[3]);
-                    acc[4] = fmaf(s, bf16_lo(sv[part].z), acc[4]);
-                    acc[5] = fmaf(s, bf16_hi(sv[part].z), acc[5]);
-                    acc[6] = fmaf(s, bf16_lo(sv[part].w), acc[6]);
-                    acc[7] = fmaf(s, bf16_hi(sv[part].w), acc[7]);
-                }
-            }
+            for (int p = 0; p < 4; ++p)
+                if (4 + p < shared_parts)
+                    sv[p] = *reinterpret_cast<const uint4 *>(
+                        shared_y + ((size_t)(4 + p) * T + t) * H + h);
+#pragma unroll
+            for (int p = 0; p < 4; ++p)
+                if (4 + p < shared_parts)
+                    accumulate8(acc, s, sv[p]);
         }
         uint4 o;
         __nv_bfloat162 p;
@@ -108,8 +114,18 @@ cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, int ro
     const size_t cap = (size_t)sm_count() * 8;
     if (blocks > cap)
         blocks = cap;
-    return launch_pdl(combine_kernel, dim3((unsigned)blocks), dim3(CB_THREADS), 0, s, y, routed_parts,
-                      inv_perm, topk_w, shared_y, shared_parts, shared_scale, T, c.hidden, c.top_k, out);
+#define MOE_CB_LAUNCH(KP)                                                                        \
+    return launch_pdl(combine_kernel<KP>, dim3((unsigned)blocks), dim3(CB_THREADS), 0, s, y,     \
+                      routed_parts, inv_perm, topk_w, shared_y, shared_parts, shared_scale, T,   \
+                      c.hidden, c.top_k, out)
+    if (c.top_k <= 2)
+        MOE_CB_LAUNCH(2);
+    if (c.top_k <= 4)
+        MOE_CB_LAUNCH(4);
+    if (c.top_k <= 8)
+        MOE_CB_LAUNCH(8);
+    MOE_CB_LAUNCH(16);
+#undef MOE_CB_LAUNCH
 }
 
 }  // namespace moe

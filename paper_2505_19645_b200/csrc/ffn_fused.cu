@@ -1060,6 +1060,8 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
 
 // ---- gather of the token rows into sorted order (B operand of the gate/up pass) ---------
 
+constexpr int GATHER_UNROLL = 4;
+
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__restrict__ perm, int A,
                    int H, int top_k, __nv_bfloat16 *__restrict__ x_sorted)
@@ -1069,24 +1071,25 @@ gather_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__restric
     const int vec_per_row = H >> 3;
     const size_t total = (size_t)A * vec_per_row;
     const size_t stride = (size_t)gridDim.x * blockDim.x;
-    // four independent row pieces per thread and pass: few CTAs (they must leave room for
-    // the FFN CTAs that start beside them) still keep enough loads in flight
-    for (size_t i0 = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i0 < total; i0 += 4 * stride) {
-        int r[4], v[4], t[4];
-        uint4 d[4];
+    // GATHER_UNROLL independent row pieces per thread and pass: few CTAs (they must leave room
+    // for the FFN CTAs that start beside them) still keep enough loads in flight
+    for (size_t i0 = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i0 < total;
+         i0 += GATHER_UNROLL * stride) {
+        int r[GATHER_UNROLL], v[GATHER_UNROLL], t[GATHER_UNROLL];
+        uint4 d[GATHER_UNROLL];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < GATHER_UNROLL; ++u) {
             const size_t i = i0 + u * stride;
             r[u] = i < total ? (int)(i / vec_per_row) : -1;
             v[u] = i < total ? (int)(i - (size_t)r[u] * vec_per_row) : 0;
             t[u] = r[u] >= 0 ? perm[r[u]] / top_k : 0;
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
+        for (int u = 0; u < GATHER_UNROLL; ++u)
             if (r[u] >= 0)
                 d[u] = reinterpret_cast<const uint4 *>(x + (size_t)t[u] * H)[v[u]];
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
+        for (int u = 0; u < GATHER_UNROLL; ++u)
             if (r[u] >= 0)
                 reinterpret_cast<uint4 *>(x_sorted + (size_t)r[u] * H)[v[u]] = d[u];
     }
@@ -1098,7 +1101,10 @@ cudaError_t launch_gather_rows(const moe_config_t &c, const __nv_bfloat16 *x, co
     const int A = T * c.top_k;
     const size_t total = (size_t)A * (c.hidden >> 3);
     size_t blocks = (total + 255) / 256;
-    const size_t cap = (size_t)sm_count() * 2;
+    // A small gather is a matter of latency: two CTAs per SM leave room for the FFN CTAs that
+    // start beside them.  A large one needs the SMs' full thread count to hide the two
+    // dependent loads of every row piece.
+    const size_t cap = (size_t)sm_count() * (total * 16 <= (4u << 20) ? 2 : 8);
     if (blocks > cap)
         blocks = cap;
     return launch_pdl(gather_rows_kernel, dim3((unsigned)blocks), dim3(256), 0, s, x, perm, A,

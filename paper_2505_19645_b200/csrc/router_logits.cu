@@ -164,9 +164,9 @@ cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
     const bool gate_row = shared_scale != nullptr && c.shared_gate && c.shared_inter > 0;
     const int n_rows = c.n_experts + (gate_row ? 1 : 0);
     const int e_tiles = (n_rows + 15) / 16;
-    // the smallest token tile that keeps the grid within about two waves
+    // the smallest token tile that keeps the grid within one wave (a CTA of 16 warps fills an SM)
     int nch = 1;
-    while (nch < 8 && (long long)e_tiles * ((T + 8 * nch - 1) / (8 * nch)) > 2LL * sm_count())
+    while (nch < 8 && (long long)e_tiles * ((T + 8 * nch - 1) / (8 * nch)) > (long long)sm_count())
         nch *= 2;
     dim3 grid(e_tiles, (T + 8 * nch - 1) / (8 * nch));
     const __nv_bfloat16 *w_sg = static_cast<const __nv_bfloat16 *>(w.w_shared_gate);
