@@ -133,7 +133,7 @@ PlanView plan_view(char *ws, const Workspace &L)
 {
     return PlanView{reinterpret_cast<int32_t *>(ws + L.plan_header),
                     reinterpret_cast<Segment *>(ws + L.plan_seg),
-                    reinterpret_cast<int32_t *>(ws + L.plan_pairs),
+                    reinterpret_cast<PairEntry *>(ws + L.plan_pairs),
                     reinterpret_cast<int32_t *>(ws + L.plan_done),
                     reinterpret_cast<int32_t *>(ws + L.plan_done) + L.plan_done_shared_at};
 }

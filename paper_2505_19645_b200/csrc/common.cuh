@@ -29,10 +29,18 @@ struct Segment {
 // plan header (ints): [0] number of segments over all activated experts,
 //                     [1] number of segment pairs (segments 2q and 2q+1 of a group form a pair),
 //                     [2], [3] routed work claimed so far by the gate/up and the down pass
+// A pair of segments (2q, 2q+1) of one group, with the group itself: everything a CTA needs to
+// start on a (pair, tile) item in one 32-byte load.
+struct __align__(16) PairEntry {
+    int32_t expert, row0, n, first_seg;  // the group (as in Segment)
+    int32_t seg;                         // plan index of the pair's first segment
+    int32_t pad[3];
+};
+
 struct PlanView {
     int32_t *header;      // written by the plan; [2], [3] advanced by the FFN kernels
     Segment *seg;         // capacity max_segments()
-    int32_t *pair_first;  // plan index of every pair's first segment, capacity max_segments()
+    PairEntry *pairs;     // one entry per pair of segments, capacity max_segments()
     // Progress of the gate/up pass, read by the down pass: 16-row units of h written so far
     // (counted once per epilogue warp) for every routed segment [max_segments()] and for
     // every 128-row segment of the shared expert [max_shared_segments()].
@@ -61,7 +69,7 @@ struct Workspace {
     size_t inv_perm;      // i32 [A]
     size_t plan_header;   // i32 [PLAN_HEADER_INTS]
     size_t plan_seg;      // Segment[max_segments]
-    size_t plan_pairs;    // i32 [max_segments]
+    size_t plan_pairs;    // PairEntry [max_segments]
     size_t plan_done;     // i32 [max_segments + max_shared_segments]
     size_t plan_done_shared_at;  // index of the shared expert's counters inside plan_done
     size_t x_sorted;      // bf16 [A, H]      token rows in sorted order
@@ -107,7 +115,7 @@ inline Workspace workspace_layout(const moe_config_t &c, int T)
     w.inv_perm = take(A * 4);
     w.plan_header = take(PLAN_HEADER_INTS * 4);
     w.plan_seg = take(sizeof(Segment) * (size_t)max_segments((int)E, (int)A));
-    w.plan_pairs = take(4 * (size_t)max_segments((int)E, (int)A));
+    w.plan_pairs = take(sizeof(PairEntry) * (size_t)max_segments((int)E, (int)A));
     w.plan_done = take(4 * ((size_t)max_segments((int)E, (int)A) + max_shared_segments(T)));
     w.plan_done_shared_at = (size_t)max_segments((int)E, (int)A);
     w.x_sorted = take(A * H * 2);

@@ -66,7 +66,7 @@ struct FfnArgs {
     int out_ld[2];
     const int32_t *plan_header;  // [0] = number of segments, [1] = number of segment pairs
     const Segment *seg;
-    const int32_t *pair_first;   // plan index of every pair's first segment
+    const PairEntry *pairs;      // the segment pairs with their groups
     int32_t *claim_counter;      // grid-wide: next unclaimed routed position / item of this pass
     int32_t *done[2];            // per segment of each group kind: 16-column units of h finished
                                  // by the gate/up pass, summed over its four epilogue warps
@@ -413,17 +413,23 @@ struct ItemWalk {
                           : (long long)nseg_total * R0;
         synced = true;
     }
-    // Claims the next chunk from the grid-wide counter (claimer only).
+    // Claims the next chunk from the grid-wide counter (claimer only).  In round-robin mode
+    // the first item of every CTA is fixed -- item gridDim.x - 1 - blockIdx.x, so that the CTAs
+    // without a shared-expert tile (the high ones) take the first routed items -- and costs no
+    // round trip to the counter; the counter hands out the items from gridDim.x on.
     __device__ void claim(int &lo, int &hi)
     {
-        int size = 1;
-        if (!a.round_robin) {
+        if (a.round_robin) {
+            lo = n_pub == 0 ? (int)(gridDim.x - 1 - blockIdx.x)
+                            : (int)gridDim.x + atomicAdd(a.claim_counter, 1);
+            hi = lo + 1;
+        } else {
             const long long left = P - *reinterpret_cast<volatile int32_t *>(a.claim_counter);
             const long long guided = left / (3 * (long long)gridDim.x);
-            size = (int)(guided > max_units ? guided : max_units);
+            const int size = (int)(guided > max_units ? guided : max_units);
+            lo = atomicAdd(a.claim_counter, size);
+            hi = (int)(lo + (long long)size < P ? lo + size : P);
         }
-        lo = atomicAdd(a.claim_counter, size);
-        hi = (int)(lo + (long long)size < P ? lo + size : P);
         if (lo >= P)
             lo = hi = -1;
     }
@@ -437,8 +443,14 @@ struct ItemWalk {
         Segment grp = sg;
         claim(lo, hi);
         if (lo >= 0 && a.round_robin) {
-            sidx = a.pair_first[lo / (ntiles * a.routed_ksplit)];
-            grp = a.seg[sidx];
+            // the pair entry carries its group: one load level between the claim and the tile
+            const int4 *pe = reinterpret_cast<const int4 *>(a.pairs + lo / (ntiles * a.routed_ksplit));
+            const int4 g = pe[0];
+            sidx = pe[1].x;
+            grp.expert = g.x;
+            grp.row0 = g.y;
+            grp.n = g.z;
+            grp.first_seg = g.w;
         }
         if (!mbar_wait(ring.empty0 + 8u * slot, par ^ 1u, ring.abort_flag, ring.status))
             return false;
@@ -469,9 +481,10 @@ struct ItemWalk {
         int *e = ring.data + slot * FF_CLAIM_WORDS;
         if (claimer) {
             for (;;) {
+                // (the counter is only read where the answer can be yes)
+                const long long ample = 4 * (long long)gridDim.x * (a.round_robin ? 1 : max_units);
                 const bool plenty =
-                    P - *reinterpret_cast<volatile int32_t *>(a.claim_counter) >
-                    4 * (long long)gridDim.x * (a.round_robin ? 1 : max_units);
+                    P > ample && P - *reinterpret_cast<volatile int32_t *>(a.claim_counter) > ample;
                 if (end_published || n_pub >= n_claims + (plenty ? 2 : 1))
                     break;
                 if (!publish_one())
@@ -1294,7 +1307,7 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
     a.out_ld[1] = c.shared_inter;
     a.plan_header = plan.header;
     a.seg = plan.seg;
-    a.pair_first = plan.pair_first;
+    a.pairs = plan.pairs;
     a.claim_counter = plan.header + 2;
     a.done[0] = plan.done_routed;
     a.done[1] = plan.done_shared;
@@ -1403,7 +1416,7 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
     a.out_ld[0] = a.out_ld[1] = c.hidden;
     a.plan_header = plan.header;
     a.seg = plan.seg;
-    a.pair_first = plan.pair_first;
+    a.pairs = plan.pairs;
     a.claim_counter = plan.header + 3;
     a.done[0] = plan.done_routed;
     a.done[1] = plan.done_shared;

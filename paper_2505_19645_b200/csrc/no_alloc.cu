@@ -53,7 +53,7 @@ static Workspace static_scratch_layout(const moe_config_t &c, int T)
     w.status = take(64 * 4);
     w.plan_header = take(PLAN_HEADER_INTS * 4);
     w.plan_seg = take(sizeof(Segment) * (size_t)max_segments(c.n_experts, (int)A));
-    w.plan_pairs = take(4 * (size_t)max_segments(c.n_experts, (int)A));
+    w.plan_pairs = take(sizeof(PairEntry) * (size_t)max_segments(c.n_experts, (int)A));
     w.plan_done = take(4 * ((size_t)max_segments(c.n_experts, (int)A) + max_shared_segments(T)));
     w.plan_done_shared_at = (size_t)max_segments(c.n_experts, (int)A);
     w.x_sorted = take(A * (size_t)c.hidden * 2);

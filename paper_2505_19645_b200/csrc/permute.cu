@@ -88,8 +88,16 @@ __device__ void build_plan(const int *cnt_sh, const int *off_sh, int *scan, int 
         scan[tid] = npair;
     __syncthreads();
     block_exclusive_scan(scan, tmp, E, total);
-    for (int q = 0; q < npair; ++q)
-        plan.pair_first[scan[tid] + q] = first + 2 * q;
+    for (int q = 0; q < npair; ++q) {
+        PairEntry pe;
+        pe.expert = tid;
+        pe.row0 = row0;
+        pe.n = cnt;
+        pe.first_seg = first;
+        pe.seg = first + 2 * q;
+        pe.pad[0] = pe.pad[1] = pe.pad[2] = 0;
+        plan.pairs[scan[tid] + q] = pe;
+    }
     if (tid == 0) {
         plan.header[1] = *total;
         plan.header[2] = 0;  // work claimed so far by the gate/up pass ...
