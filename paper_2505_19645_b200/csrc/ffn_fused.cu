@@ -1050,9 +1050,11 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             if (lane == 0) {
                 mbar_arrive(acc_empty(buf));
                 if (GATED) {
-                    // publish: this warp's part of the tile is in h
-                    __threadfence();
-                    atomicAdd(args.done[it.grp] + it.seg, it.h >> 4);
+                    // publish: this warp's part of the tile is in h (a releasing reduction: the
+                    // warp does not wait for its stores to become visible, the counter does)
+                    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(args.done[it.grp] + it.seg),
+                                 "r"(it.h >> 4)
+                                 : "memory");
                 }
             }
         }
