@@ -103,6 +103,24 @@ def test_row_permutation_equivariance():
     assert torch.equal(out_p, out[p])
 
 
+def test_layer_parity_with_plain_stream_ordering():
+    """MOE_NO_PDL=1 (read once per process) launches every kernel with plain stream ordering:
+    the kernels then run one after the other and every progress counter is complete when its
+    reader starts.  Runs a few of the cases above in a child process."""
+    import os
+    import subprocess
+    import sys
+
+    env = dict(os.environ, MOE_NO_PDL="1")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run(
+        [sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_layer.py"), "-q", "-x",
+         "-m", "gpu", "-k", "small_shapes and (qwen-like or mixtral-like or ksplit-routed)"],
+        env=env, cwd=root, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+    assert "passed" in r.stdout
+
+
 # ---- full-size shapes in the launch configuration the benchmark times -------------------
 # The oracle evaluates a seeded sample of token rows (the layer is token-wise, so a row
 # check is exact); routing and grouping are checked on every token.
