@@ -22,6 +22,27 @@ int sm_count()
     return cached[dev];
 }
 
+void prefer_max_shared_carveout(const void *kernel)
+{
+    // a handful of kernels: a small table of those already configured (a race between two
+    // threads at worst sets the attribute twice)
+    struct Key {
+        const void *kernel;
+        int device;
+    };
+    static Key seen[256];
+    static int n_seen = 0;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    for (int i = 0; i < n_seen; ++i)
+        if (seen[i].kernel == kernel && seen[i].device == dev)
+            return;
+    cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                         cudaSharedmemCarveoutMaxShared);
+    if (n_seen < 256)
+        seen[n_seen++] = Key{kernel, dev};
+}
+
 // MOE_NO_PDL=1 in the environment launches every kernel with plain stream ordering.
 bool pdl_enabled()
 {

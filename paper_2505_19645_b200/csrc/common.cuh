@@ -204,6 +204,13 @@ moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_b
 // ---------------------------------------------------------------------------------------
 #ifdef __CUDACC__
 
+// An SM changes its L1 / shared-memory split only while it is idle.  The FFN kernels need the
+// largest shared-memory split; if the small kernels before them ran with another one, an FFN
+// CTA could not start on an SM as long as one of their CTAs is resident there (measured: the
+// gate/up pass began only when the row gather had finished).  So every kernel of the library
+// asks for the same, largest split (once per kernel).
+void prefer_max_shared_carveout(const void *kernel);
+
 // Launch with the programmatic-stream-serialization attribute: the kernel may begin while its
 // predecessor in the stream is still running and must execute griddepcontrol.wait before it
 // touches anything the predecessor produces.
@@ -211,6 +218,7 @@ template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
                               cudaStream_t s, Args &&...args)
 {
+    prefer_max_shared_carveout(reinterpret_cast<const void *>(kernel));
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
     cfg.blockDim = block;

@@ -1075,7 +1075,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
 
 // ---- gather of the token rows into sorted order (B operand of the gate/up pass) ---------
 
-constexpr int GATHER_UNROLL = 4;
+constexpr int GATHER_UNROLL = 8;
 
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__restrict__ perm, int A,
@@ -1086,8 +1086,7 @@ gather_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__restric
     const int vec_per_row = H >> 3;
     const size_t total = (size_t)A * vec_per_row;
     const size_t stride = (size_t)gridDim.x * blockDim.x;
-    // GATHER_UNROLL independent row pieces per thread and pass: few CTAs (they must leave room
-    // for the FFN CTAs that start beside them) still keep enough loads in flight
+    // GATHER_UNROLL independent row pieces per thread and pass
     for (size_t i0 = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i0 < total;
          i0 += GATHER_UNROLL * stride) {
         int r[GATHER_UNROLL], v[GATHER_UNROLL], t[GATHER_UNROLL];
@@ -1115,11 +1114,15 @@ cudaError_t launch_gather_rows(const moe_config_t &c, const __nv_bfloat16 *x, co
 {
     const int A = T * c.top_k;
     const size_t total = (size_t)A * (c.hidden >> 3);
-    size_t blocks = (total + 255) / 256;
-    // A small gather is a matter of latency: two CTAs per SM leave room for the FFN CTAs that
-    // start beside them.  A large one needs the SMs' full thread count to hide the two
+    // An FFN CTA does not start on an SM while a CTA of another kernel is resident there
+    // (measured, whatever their shared-memory and register needs), so until this kernel has
+    // finished the gate/up pass runs its shared-expert tiles only on the SMs this kernel
+    // leaves alone.  Up to 16 MB of rows the gather therefore runs as one CTA per SM at most
+    // (the hardware places them on about half of the SMs; fewer, larger CTAs made the gather
+    // itself too slow); a large gather needs every SM's full thread count to hide the two
     // dependent loads of every row piece.
-    const size_t cap = (size_t)sm_count() * (total * 16 <= (4u << 20) ? 2 : 8);
+    size_t blocks = (total + 255) / 256;
+    const size_t cap = (size_t)sm_count() * (total * 16 <= (16u << 20) ? 1 : 8);
     if (blocks > cap)
         blocks = cap;
     return launch_pdl(gather_rows_kernel, dim3((unsigned)blocks), dim3(256), 0, s, x, perm, A,
