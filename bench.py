@@ -310,7 +310,7 @@ def main():
                     help="sweep the config's (B, gamma) grid or the 19 batch sizes x gamma 0/2/4")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--sweep-steps", type=int, default=10)
+    ap.add_argument("--sweep-steps", type=int, default=30)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -410,6 +410,7 @@ def main():
                     base_ms = med
                 roof = layer_roof_ms(Ti, na)
                 sweep.append({"B": Bi, "gamma": gi, "T": Ti, "us": round(med * 1e3, 2),
+                              "us_min": round(min(ms) * 1e3, 2),
                               "tokens_per_s": round(Ti / (med * 1e-3), 1), "n_active": na,
                               "n_active_expected": round(expected_active(shape.n_experts, shape.top_k, Ti), 2),
                               "roof_us": round(roof * 1e3, 2), "roof_frac": round(roof / med, 4),
