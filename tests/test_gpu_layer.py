@@ -32,6 +32,11 @@ def test_tiny_config_full_parity():
     ("ksplit-routed", 256, 4, 2, 4096, 0, 0, 1, 0, 10, 3, None),       # four planes of y
     ("ksplit-odd", 384, 8, 2, 2176, 0, 0, 1, 0, 3, 2, None),           # two chunks, ragged second
     ("dense-contrast", 256, 1, 1, 3072, 3072, 0, 0, 1, 65, 1, None),   # E = k = 1, 130 rows
+    # small batches (one routing launch) at the expert counts that select other code paths
+    ("dsv3-like-small", 1024, 256, 8, 256, 256, 1, 1, 0, 4, 3, None),  # 16 tokens, 256 experts
+    ("e512-small", 256, 512, 4, 128, 0, 0, 1, 0, 5, 1, 1.0),           # the expert limit, skewed
+    ("e24-32tok", 256, 24, 16, 128, 128, 0, 0, 1, 8, 3, None),         # 32 tokens x top-16: 512 assignments
+    ("e24-33tok", 256, 24, 16, 128, 128, 0, 0, 1, 11, 2, None),        # one token more: the long chain
 ])
 def test_layer_parity_small_shapes(name, H, E, k, I, Is, score, renorm, sgate, B, gamma, zipf):
     shape = wl.small_shape(name, H, E, k, I, Is, score, renorm, sgate)
