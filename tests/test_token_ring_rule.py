@@ -1,0 +1,106 @@
+"""Model of the FFN kernels' token ring (CPU only).
+
+The token-operand ring of `ffn_fused_kernel` holds entries of 2 KB units that never wrap: an
+entry that does not fit before the end of the ring starts at unit 0, and the producer may place
+entry j once everything before the oldest entry still in use is free.  The MMA side consumes
+the entries of one k step together (one entry, or two for a pair of segments).  This test
+replays that rule over random item sequences: the geometries the host chooses (48 units with
+pairs of segments, 16 units without) never stall and never overlap live entries, and a ring
+of exactly two full entries with pairs does stall -- which is why the host refuses it.
+"""
+import random
+
+ENTRIES = 8  # barrier pairs = entries in flight
+
+
+def replay(units, steps):
+    """steps: list of lists of entry sizes consumed together.  Returns 'ok', 'stall' or
+    'overlap'."""
+    seq = [m for st in steps for m in st]
+    first_of_step = []
+    acc = 0
+    for st in steps:
+        first_of_step.append(acc)
+        acc += len(st)
+    cur = 0          # next free physical unit
+    v_cur = 0        # virtual position issued up to (physical position + laps * units)
+    v_rel = 0        # virtual position free up to
+    released = 0     # entries the producer knows to be consumed
+    v_start = {}     # virtual start of every issued entry's rows
+    live = {}        # entry -> (physical start, size), until released
+    issued = consumed_entries = consumed_steps = 0
+    while consumed_steps < len(steps):
+        progressed = False
+        if issued < len(seq):
+            j, m = issued, seq[issued]
+            pad, at = 0, cur
+            if at + m > units:
+                pad, at = units - cur, 0
+            start, end = v_cur + pad, v_cur + pad + m
+            rel, vr = released, v_rel
+            blocked = False
+            while rel < j and (j - rel >= ENTRIES or end - vr > units):
+                if rel < consumed_entries:   # its MMAs have completed
+                    rel += 1
+                    vr = v_start[rel] if rel < j else start
+                else:
+                    blocked = True
+                    break
+            released, v_rel = rel, vr
+            for q in [q for q in live if q < released]:
+                del live[q]
+            if not blocked:
+                for a2, m2 in live.values():
+                    if not (at + m <= a2 or a2 + m2 <= at):
+                        return "overlap"
+                live[j] = (at, m)
+                v_start[j] = start
+                v_cur, cur = end, at + m
+                issued += 1
+                progressed = True
+        s = consumed_steps
+        if first_of_step[s] + len(steps[s]) <= issued:
+            consumed_entries += len(steps[s])
+            consumed_steps += 1
+            progressed = True
+        if not progressed:
+            return "stall"
+    return "ok"
+
+
+def random_steps(rng, max_pieces, pairs):
+    """Items as the kernels produce them: a full first segment (16 units at two k boxes per
+    slot) with any second segment, or a single segment; sizes are even (two k boxes)."""
+    steps = []
+    for _ in range(rng.randint(1, 8)):
+        k_steps = rng.randint(1, 6)
+        if pairs and rng.random() < 0.5:
+            steps += [[2 * max_pieces, 2 * rng.randint(1, max_pieces)]] * k_steps
+        else:
+            steps += [[2 * rng.randint(1, max_pieces)]] * k_steps
+    return steps
+
+
+def test_ring_of_three_full_entries_never_stalls_with_pairs():
+    rng = random.Random(1)
+    for _ in range(4000):
+        assert replay(48, random_steps(rng, 8, True)) == "ok"
+
+
+def test_small_ring_never_stalls_without_pairs():
+    rng = random.Random(2)
+    for _ in range(4000):
+        assert replay(16, random_steps(rng, 4, False)) == "ok"
+
+
+def test_ring_of_two_full_entries_can_stall_with_pairs():
+    # a 16-unit entry that sits at unit 10 leaves no room for its 14-unit partner
+    assert replay(32, [[10]] * 4 + [[16, 14]] * 2) == "stall"
+    rng = random.Random(3)
+    outcomes = {replay(32, random_steps(rng, 8, True)) for _ in range(2000)}
+    assert "overlap" not in outcomes and "stall" in outcomes
+
+
+def test_entries_in_flight_are_bounded_by_the_barrier_pairs():
+    # many tiny entries: the eight barrier pairs, not the space, limit the producer
+    assert replay(48, [[2]] * 100) == "ok"
