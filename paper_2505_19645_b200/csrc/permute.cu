@@ -285,6 +285,90 @@ route_group_small_kernel(const float *__restrict__ logits, const __nv_bfloat16 *
     }
     __syncthreads();
 
+    if (A <= 32) {
+        // At most a warp's worth of assignments: one warp sorts them with shuffles and every
+        // thread derives its expert's table entries from the (few) assignments directly --
+        // two barriers in all instead of the scans below.
+        if (warp == 0) {
+            const int e = lane < A ? expert_of[lane] : -1;
+            const uint32_t peers = __match_any_sync(0xffffffffu, e);
+            const int rank = __popc(peers & ((1u << lane) - 1u));
+            int less = 0;
+#pragma unroll
+            for (int src = 0; src < 32; ++src) {
+                const int other = __shfl_sync(0xffffffffu, e, src);
+                less += (other >= 0 && other < e) ? 1 : 0;
+            }
+            flag[lane] = (e >= 0 && lane == __ffs(peers) - 1) ? 1 : 0;  // first of its expert
+            if (e >= 0) {
+                const int pos = less + rank;  // stable: ascending assignment id inside an expert
+                token_of[pos] = lane / k;
+                if (blockIdx.x == 0) {
+                    perm[pos] = lane;
+                    inv_perm[lane] = pos;
+                }
+            }
+        }
+        __syncthreads();
+        if (blockIdx.x == 1) {
+            int cnt = 0, off = 0, arank = 0, n_act = 0;
+            for (int a = 0; a < A; ++a) {
+                const int ea = expert_of[a];
+                cnt += ea == tid ? 1 : 0;
+                off += ea < tid ? 1 : 0;
+                arank += (flag[a] && ea < tid) ? 1 : 0;  // activated experts below this one
+                n_act += flag[a];
+            }
+            if (tid < E) {
+                counts[tid] = cnt;
+                offsets[tid] = off;
+                if (tid >= n_act)
+                    active[tid] = -1;
+                if (cnt > 0) {
+                    active[arank] = tid;
+                    if (plan.header != nullptr) {  // one segment and one pair per activated expert
+                        Segment sg;
+                        sg.expert = tid;
+                        sg.row0 = off;
+                        sg.n = cnt;
+                        sg.first_seg = arank;
+                        plan.seg[arank] = sg;
+                        plan.done_routed[arank] = 0;
+                        PairEntry pe;
+                        pe.expert = tid;
+                        pe.row0 = off;
+                        pe.n = cnt;
+                        pe.first_seg = arank;
+                        pe.seg = arank;
+                        pe.pad[0] = pe.pad[1] = pe.pad[2] = 0;
+                        plan.pairs[arank] = pe;
+                    }
+                }
+            }
+            if (tid == 0) {
+                offsets[E] = A;
+                n_active[0] = n_act;
+                if (plan.header != nullptr) {
+                    plan.header[0] = n_act;  // segments
+                    plan.header[1] = n_act;  // pairs
+                    plan.header[2] = 0;
+                    plan.header[3] = 0;
+                    status[0] = 0;
+                }
+            }
+        } else if (blockIdx.x >= 2) {
+            const int vec_per_row = H >> 3;
+            const int n_copy = gridDim.x - 2;
+            for (int r = blockIdx.x - 2; r < A; r += n_copy) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)token_of[r] * H);
+                uint4 *dst = reinterpret_cast<uint4 *>(x_sorted + (size_t)r * H);
+                for (int v = tid; v < vec_per_row; v += PERM_THREADS)
+                    dst[v] = src[v];
+            }
+        }
+        return;
+    }
+
     // counting sort, one assignment per thread (threads beyond A idle along)
     const bool few = E <= 32;
     const int my_e = tid < A ? expert_of[tid] : -1;

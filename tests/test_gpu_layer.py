@@ -35,6 +35,8 @@ def test_tiny_config_full_parity():
     # small batches (one routing launch) at the expert counts that select other code paths
     ("dsv3-like-small", 1024, 256, 8, 256, 256, 1, 1, 0, 4, 3, None),  # 16 tokens, 256 experts
     ("e512-small", 256, 512, 4, 128, 0, 0, 1, 0, 5, 1, 1.0),           # the expert limit, skewed
+    ("e512-warp", 256, 512, 4, 128, 128, 1, 1, 0, 2, 3, 1.0),          # 32 assignments: sorted by one warp
+    ("e8-warp-dup", 128, 8, 2, 256, 0, 0, 1, 0, 3, 4, None),           # 30 assignments on 8 experts
     ("e24-32tok", 256, 24, 16, 128, 128, 0, 0, 1, 8, 3, None),         # 32 tokens x top-16: 512 assignments
     ("e24-33tok", 256, 24, 16, 128, 128, 0, 0, 1, 11, 2, None),        # one token more: the long chain
 ])
