@@ -14,20 +14,26 @@
 //
 // Work partition.  Output features are independent, so the weight rows of all routed
 // groups are laid end to end (one position = 16 rows of one group for one of its 128-row
-// segments) and every CTA of the persistent grid takes one contiguous range: no tile-count
-// quantisation, no tail wave.  The shared expert's rows are cut into full-height tiles that
+// segments) and the CTAs of the persistent grid claim chunks of positions at run time from a
+// grid-wide counter (chunk ends on tile boundaries, sizes shrinking as the work runs out), or,
+// where chunks would be too short or too many, single (segment pair, tile, k chunk) items: a
+// CTA that starts late or runs slowly takes less, there is no tile-count quantisation and no
+// tail wave.  The shared expert's rows are cut into (tile, k chunk, segment pair) units that
 // are dealt round-robin to the CTAs; they depend on nothing the layer computes, so they run
-// before the routing result exists, and the routed ranges are then sized so that
-// shared + routed cost is level across the grid.  Inside its range a CTA cuts tiles of at
-// most 128 (gate/up) or 256 (down) rows.  A group with more than 128 token rows has several
-// segments; two segments share one pass over a tile (the weight slot is multiplied with
-// both, one accumulator buffer each), and the shared expert's (tile, segment pair) units are
-// spread over the CTAs so that the units of one tile run at the same time and meet in L2.
+// before the routing result exists.  Tiles have at most 128 (gate/up) or 256 (down) rows.  A
+// group with more than 128 token rows has several segments; two segments share one pass over
+// a tile (the weight slot is multiplied with both, one accumulator buffer each), and the
+// units of one shared tile run at the same time on neighbouring CTAs and meet in L2.
+//
+// Between the passes.  The gate/up pass counts, per segment, the 16-column units of h its
+// epilogue warps have stored (a releasing reduction); the down pass starts while the gate/up
+// pass is still running and fetches a segment's rows of h once the segment's count is
+// complete (acquire load, then a proxy fence before the TMA loads).
 //
 // A weight slot of the shared-memory ring holds two 64-element k boxes of one tile (64 KB
 // for a full tile), so that one producer/consumer hand-shake moves enough bytes to keep HBM
-// busy and every weight row is requested in 256 contiguous bytes; the token operand lives in a second ring whose entries are sized
-// by the segment's row count.
+// busy and every weight row is requested in 256 contiguous bytes; the token operand lives in
+// a second ring whose entries are sized by the segment's row count and never wrap.
 //
 // CTA = 7 warps.  warp 0: weight producer (one lane issues TMA), warp 1: MMA issuer (one
 // lane) and owner of the TMEM allocation, warp 2: token-operand producer, warps 3..6:
@@ -39,7 +45,8 @@
 // Programmatic dependent launch: the kernels may start while their predecessor in the stream
 // is still running.  Work that depends only on the caller's inputs (shared-expert tiles in the
 // gate/up pass, weight prefetch in the down pass) is done before griddepcontrol.wait, so it
-// overlaps the routing kernels; everything produced inside the layer is touched after it.
+// overlaps the routing kernels; everything produced inside the layer is touched after it,
+// except h, which the down pass takes segment by segment as described above.
 #include <cuda.h>
 #include <math.h>
 #include <stdlib.h>
