@@ -22,6 +22,9 @@ __device__ __forceinline__ void warp_route_topk(const float *__restrict__ z, int
     for (int i = 0; i < VPL; ++i) {
         const int e = lane + 32 * i;
         v[i] = e < E ? z[e] : -FLT_MAX;
+        if (!(v[i] == v[i]))
+            v[i] = -FLT_MAX;  // NaN (outside the contract) ranks lowest: the arg-max below needs
+                              // a total order for all lanes to agree, else an index could be lost
         vmax = fmaxf(vmax, v[i]);
     }
 #pragma unroll

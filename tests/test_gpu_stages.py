@@ -41,6 +41,37 @@ def test_route_topk_bit_exact(E, k, score_fn, renorm):
     assert np.abs(w.cpu().numpy().astype(np.float64) - w_ref).max() <= GATE_W_ATOL * shape.routed_scale
 
 
+@pytest.mark.parametrize("E,k", [(8, 2), (60, 4), (256, 8)])
+def test_route_topk_stays_in_bounds_on_non_finite_logits(E, k):
+    """Logits are finite by contract; NaN / Inf rows may come out in any order, but the
+    selection must still be k distinct experts inside [0, E): nothing downstream indexes out
+    of bounds."""
+    api = _api()
+    T = 64
+    rng = np.random.default_rng(E + k)
+    z = rng.normal(0, 1, size=(T, E)).astype(np.float32)
+    z[0, :] = np.nan
+    z[1, ::2] = np.nan
+    z[2, :] = -np.inf
+    z[3, :] = np.inf
+    z[4, 0] = np.nan
+    z[5, -1] = np.inf
+    z[6, : E // 2] = -np.inf
+    shape = wl.small_shape("nf", 64, E, k, 64, 0, 0, 1, 0)
+    cfg = api.make_config(shape)
+    idx = torch.full((T, k), -7, dtype=torch.int32, device="cuda")
+    w = torch.empty((T, k), dtype=torch.float32, device="cuda")
+    api.moe_route_topk(cfg, torch.from_numpy(z).cuda(), idx, w)
+    torch.cuda.synchronize()
+    got = idx.cpu().numpy()
+    assert got.min() >= 0 and got.max() < E
+    for t in range(T):
+        assert len(set(got[t].tolist())) == k
+    # finite rows are unaffected by their neighbours
+    idx_ref, _ = oracle.route_topk(z[7:], k, 0, 1, 1.0)
+    np.testing.assert_array_equal(got[7:], idx_ref)
+
+
 @pytest.mark.parametrize("T,k,E,mode", [
     (1, 2, 8, "rand"), (16, 2, 8, "rand"), (640, 4, 60, "rand"), (1280, 8, 64, "rand"),
     (4096, 8, 256, "rand"), (300, 1, 512, "rand"), (257, 4, 60, "one"), (100, 8, 8, "all"),
