@@ -187,6 +187,15 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
  * invalid but the context stays usable), or MOE_ERR_CUDA. */
 moe_status_t moe_check(void *ws, void *stream);
 
+/* Self-test of the failure path (no counterpart in the paper).  Every wait inside the kernels is
+ * bounded; when one gives up, the kernel raises the workspace's status word and returns, and
+ * moe_check reports MOE_ERR_TIMEOUT while the context stays usable.  This call enqueues one tiny
+ * kernel that runs exactly that wait -- the one the down projection uses for the progress
+ * counters of the gate/up pass -- on a word nothing ever sets, with a limit of limit_us
+ * microseconds (1 .. 1000000).  ws: any workspace of at least 256 bytes; its status word is
+ * overwritten.  Returns at once; the outcome is read with moe_check(ws, stream). */
+moe_status_t moe_selftest_wait_limit(void *ws, int32_t limit_us, void *stream);
+
 /* Measurement aid (no counterpart in the paper; its Sec. 3.3 model attributes the layer's
  * time to weight loading, which the benchmark verifies per kernel).  Every following
  * moe_verify_layer call of this thread records start_event before and stop_event after the

@@ -21,7 +21,8 @@ STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_UNSUPPORTED",
 
 EXPORTS = ["moe_workspace_bytes", "moe_router_logits", "moe_route_topk", "moe_permute",
            "moe_grouped_swiglu", "moe_combine", "moe_verify_layer", "moe_check",
-           "moe_last_launch_count", "moe_status_string", "moe_profile_stage"]
+           "moe_last_launch_count", "moe_status_string", "moe_profile_stage",
+           "moe_selftest_wait_limit"]
 
 STAGES = {"router_logits": 0, "route_topk": 1, "permute": 2, "plan": 3, "gate_up": 4, "down": 5,
           "combine": 6, "gather": 7}
@@ -88,6 +89,8 @@ def load_library():
     lib.moe_check.argtypes = [vp, vp]
     lib.moe_profile_stage.restype = i32
     lib.moe_profile_stage.argtypes = [i32, vp, vp]
+    lib.moe_selftest_wait_limit.restype = i32
+    lib.moe_selftest_wait_limit.argtypes = [vp, i32, vp]
     lib.moe_last_launch_count.restype = i32
     lib.moe_last_launch_count.argtypes = []
     lib.moe_status_string.restype = ctypes.c_char_p
@@ -256,6 +259,12 @@ def moe_verify_layer(cfg, weights, x, B: int, gamma: int, out, ws, dbg: dict | N
 
 def moe_check(ws, stream=None):
     _check(load_library().moe_check(_ptr(ws), _stream_ptr(stream)), "moe_check")
+
+
+def moe_selftest_wait_limit(ws, limit_us: int, stream=None):
+    """Enqueue the bounded-wait self-test; moe_check(ws) then raises MOE_ERR_TIMEOUT."""
+    _check(load_library().moe_selftest_wait_limit(_ptr(ws), int(limit_us), _stream_ptr(stream)),
+           "moe_selftest_wait_limit")
 
 
 def moe_profile_stage(stage, start_event=None, stop_event=None):

@@ -411,6 +411,20 @@ moe_status_t moe_check(void *ws, void *stream)
     return word == 0 ? MOE_OK : MOE_ERR_TIMEOUT;
 }
 
+moe_status_t moe_selftest_wait_limit(void *ws, int32_t limit_us, void *stream)
+{
+    if (!ws || !aligned16(ws) || limit_us < 1 || limit_us > 1000000)
+        return MOE_ERR_INVALID_ARG;
+    moe_status_t st = check_device();
+    if (st != MOE_OK)
+        return st;
+    int32_t *status = static_cast<int32_t *>(ws);  // the status region is the first of the workspace
+    int launches = 0;
+    MOE_TRY_LAUNCH(launch_wait_limit_selftest(status, status + 1, limit_us,
+                                              static_cast<cudaStream_t>(stream)));
+    return MOE_OK;
+}
+
 moe_status_t moe_profile_stage(int32_t stage, void *start_event, void *stop_event)
 {
     if (stage > MOE_STAGE_GATHER || (stage >= 0 && (!start_event || !stop_event)))

@@ -97,6 +97,7 @@ struct FfnArgs {
     int w_slot_bytes;  // capacity of a weight slot
     int n_w_slots;
     int x_units;       // token ring size in FF_X_UNIT units
+    int wait_us;       // limit of every wait inside the kernel, microseconds
 };
 
 // Tensor maps of one pass: weights [kind][matrix][box height], token operand [kind][box height].
@@ -148,8 +149,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait.  Returns false (and raises the abort flag) if the phase did not complete in
-// FF_WAIT_NS or another role already aborted.
+// Bounded wait.  Returns false (and raises the abort flag) if the phase did not complete within
+// the wait limit or another role already aborted.  abort_flag[0] is the CTA's abort flag,
+// abort_flag[1] the limit in microseconds (FF_WAIT_NS unless the host shortened it).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                           int32_t *status)
 {
@@ -163,7 +165,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
                 return true;
         if (*abort_flag)
             return false;
-        if (global_ns() - t0 > FF_WAIT_NS) {
+        if (global_ns() - t0 > 1000ull * (uint64_t)abort_flag[1]) {
             *abort_flag = 1;
             atomicExch(status, 1);
             return false;
@@ -193,7 +195,7 @@ __device__ __forceinline__ bool counter_wait(const int32_t *p, int target, volat
         }
         if (*abort_flag)
             return false;
-        if (global_ns() - t0 > FF_WAIT_NS) {
+        if (global_ns() - t0 > 1000ull * (uint64_t)abort_flag[1]) {
             *abort_flag = 1;
             atomicExch(status, 1);
             return false;
@@ -683,7 +685,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * FF_MAX_W_SLOTS + 2 * FF_X_ENTRIES + 4 + 2 * FF_CLAIMS];
     __shared__ uint32_t tmem_base_holder;
-    __shared__ int abort_flag;
+    __shared__ int abort_flag[2];  // [0] raised by the first wait that gives up, [1] wait limit (us)
     __shared__ int claim_data[FF_CLAIMS * FF_CLAIM_WORDS];
 
     const int NS = args.n_w_slots;
@@ -705,7 +707,8 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = args.wait_us;
         for (int s = 0; s < NS; ++s) {
             mbar_init(w_full(s), 1);
             mbar_init(w_empty(s), 1);
@@ -736,7 +739,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_holder;
-    volatile int *abortp = &abort_flag;
+    volatile int *abortp = abort_flag;
     const ClaimRing claims{claim_data, claim_full0, claim_empty0, abortp, args.status};
 
     if (warp == 0) {
@@ -802,12 +805,6 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 walk.sync(true);
             if (!launched)
                 griddep_launch();
-            if (!ok) {
-                // copies already issued may still be landing: give them time before teardown
-                const uint64_t t0 = global_ns();
-                while (global_ns() - t0 < 1000000ull) {
-                }
-            }
         }
     } else if (warp == 2) {
         // ---------------- token-operand producer ----------------
@@ -899,11 +896,6 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 walk.sync(true);
             if (!GATED)
                 griddep_wait();  // no kernel of the chain completes before its predecessor
-            if (!ok) {
-                const uint64_t t0 = global_ns();
-                while (global_ns() - t0 < 1000000ull) {
-                }
-            }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
@@ -1069,6 +1061,15 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             walk.sync(true);
     }
 
+    if (*abortp) {
+        // A wait gave up.  Copies and tensor-core instructions already issued may still be in
+        // flight: every thread that sees the flag (the one that raised it always does) holds
+        // the CTA for a millisecond, far longer than any of them takes, before shared memory
+        // and TMEM are given back.
+        const uint64_t t0 = global_ns();
+        while (global_ns() - t0 < 1000000ull) {
+        }
+    }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -1078,6 +1079,30 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                      "r"(FF_TMEM_COLS)
                      : "memory");
     }
+}
+
+// ---- self-test of the bounded wait ---------------------------------------------------------
+
+// Waits, with the given limit, for a progress counter that nothing advances: the wait the down
+// pass uses for the gate/up pass's counters must give up, raise the status word and return.
+__global__ void wait_limit_selftest_kernel(int32_t *status, int32_t *never_set, int limit_us)
+{
+    __shared__ int abort_flag[2];
+    if (threadIdx.x == 0) {
+        abort_flag[0] = 0;
+        abort_flag[1] = limit_us;
+        status[0] = 0;
+        never_set[0] = 0;
+        __threadfence();
+        counter_wait(never_set, 1, abort_flag, status);
+    }
+}
+
+cudaError_t launch_wait_limit_selftest(int32_t *status, int32_t *never_set, int limit_us,
+                                       cudaStream_t s)
+{
+    wait_limit_selftest_kernel<<<1, 32, 0, s>>>(status, never_set, limit_us);
+    return cudaGetLastError();
 }
 
 // ---- gather of the token rows into sorted order (B operand of the gate/up pass) ---------
@@ -1241,6 +1266,7 @@ static void ffn_geometry(int T, FfnArgs &a)
     if (ns > FF_MAX_W_SLOTS)
         ns = FF_MAX_W_SLOTS;
     a.n_w_slots = ns;
+    a.wait_us = (int)(FF_WAIT_NS / 1000ull);
 }
 
 // Range mode keeps every CTA alone on "its" groups, perfectly levelled.  It loses when

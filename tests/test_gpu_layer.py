@@ -128,6 +128,33 @@ def test_layer_parity_with_plain_stream_ordering():
     assert "passed" in r.stdout
 
 
+def test_wait_limit_expiry_is_reported_and_the_context_stays_usable():
+    """Every wait inside the kernels has a limit.  The self-test runs the down pass's wait for
+    a progress counter on a word nothing sets: it gives up after its limit, the kernel raises
+    the workspace's status word and returns, moe_check reports MOE_ERR_TIMEOUT, nothing
+    faults, and the same workspace serves a correct layer call right after."""
+    import time
+    from paper_2505_19645_b200 import api
+
+    shape = wl.small_shape("limit", 512, 60, 4, 352, 1408, 0, 0, 1)
+    w = wl.make_weights(shape, 160, "cuda")
+    x = wl.make_tokens(shape, 65, 265, "cuda")
+    cfg = api.make_config(shape)
+    ws = api.alloc_workspace(cfg, 65)
+    run_gpu_layer(shape, w, x, 13, 4, ws=ws)
+    t0 = time.perf_counter()
+    api.moe_selftest_wait_limit(ws, 20000)  # 20 ms
+    with pytest.raises(api.MoeError) as err:
+        api.moe_check(ws)
+    waited = time.perf_counter() - t0
+    assert err.value.status == 5  # MOE_ERR_TIMEOUT
+    assert 0.015 < waited < 1.0
+    out, _ = run_gpu_layer(shape, w, x, 13, 4, ws=ws)   # clears the status word, runs normally
+    ref, _ = run_gpu_layer(shape, w, x, 13, 4)
+    assert torch.equal(out, ref)
+    check_layer_against_oracle(shape, w, x, 13, 4)
+
+
 # ---- full-size shapes in the launch configuration the benchmark times -------------------
 # The oracle evaluates a seeded sample of token rows (the layer is token-wise, so a row
 # check is exact); routing and grouping are checked on every token.
