@@ -59,85 +59,15 @@ __device__ __forceinline__ void load_row8(const RowSrc &r, int k, float (&v)[8])
     }
 }
 
+// Sum of the warps' partial accumulators of one block of 16 router rows, written out.
 template <int NCH>
-__global__ void __launch_bounds__(RL_WARPS_FOR(NCH) * 32)
-router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ w_router,
-                     const float *__restrict__ bias, const __nv_bfloat16 *__restrict__ w_sg,
-                     int T, int H, int E, int n_rows, float *__restrict__ logits,
-                     float *__restrict__ shared_scale, int32_t *__restrict__ zero, int zero_n)
+__device__ __forceinline__ void reduce_and_store(const float (&part)[RL_WARPS_FOR(NCH)][NCH][4][32],
+                                                 int e0, int t0, int T, int E, int n_rows,
+                                                 const float *__restrict__ bias,
+                                                 float *__restrict__ logits,
+                                                 float *__restrict__ shared_scale)
 {
     constexpr int RL_WARPS = RL_WARPS_FOR(NCH);
-    __shared__ float part[RL_WARPS][NCH][4][32];
-    griddep_wait();    // first kernel of a layer call: everything older is complete from here on
-    if (zero != nullptr && blockIdx.x == 0 && blockIdx.y == 0) {
-        // counters that a later kernel of this call updates before the plan kernel has run
-        for (int i = threadIdx.x; i < zero_n; i += blockDim.x)
-            zero[i] = 0;
-        __threadfence();
-        __syncthreads();
-    }
-    griddep_launch();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g = lane >> 2, tq = lane & 3;
-    const int e0 = blockIdx.x * 16;
-    const int t0 = blockIdx.y * (8 * NCH);
-
-    auto row_src = [&](int e) {
-        RowSrc r{nullptr, nullptr};
-        if (e < E)
-            r.f32 = w_router + (size_t)e * H + 8 * tq;
-        else if (e == E && e < n_rows)
-            r.bf16 = w_sg + 8 * tq;
-        return r;
-    };
-    const RowSrc rlo = row_src(e0 + g), rhi = row_src(e0 + g + 8);
-    const __nv_bfloat16 *b[NCH];
-#pragma unroll
-    for (int c = 0; c < NCH; ++c)
-        b[c] = x + (size_t)min(t0 + c * 8 + g, T - 1) * H + 8 * tq;
-
-    float acc[NCH][4];
-#pragma unroll
-    for (int c = 0; c < NCH; ++c)
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-            acc[c][q] = 0.f;
-
-    const int nsteps = H >> 5;
-    const int s0 = warp * nsteps / RL_WARPS, s1 = (warp + 1) * nsteps / RL_WARPS;
-#pragma unroll 4
-    for (int s = s0; s < s1; ++s) {
-        const int k = s * 32;
-        float lo8[8], hi8[8];
-        load_row8(rlo, k, lo8);
-        load_row8(rhi, k, hi8);
-        uint4 B[NCH];
-#pragma unroll
-        for (int c = 0; c < NCH; ++c)
-            B[c] = ld_cached_v4(b[c] + k);
-        // physical k positions 8tq+{0..3} feed the first MMA, 8tq+{4..7} the second
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const Split3 a0 = split_pair(lo8[4 * half + 0], lo8[4 * half + 1]);
-            const Split3 a1 = split_pair(hi8[4 * half + 0], hi8[4 * half + 1]);
-            const Split3 a2 = split_pair(lo8[4 * half + 2], lo8[4 * half + 3]);
-            const Split3 a3 = split_pair(hi8[4 * half + 2], hi8[4 * half + 3]);
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                const uint32_t b0 = half ? B[c].z : B[c].x, b1 = half ? B[c].w : B[c].y;
-                mma_bf16_16816(acc[c], a0.lo, a1.lo, a2.lo, a3.lo, b0, b1);
-                mma_bf16_16816(acc[c], a0.mid, a1.mid, a2.mid, a3.mid, b0, b1);
-                mma_bf16_16816(acc[c], a0.hi, a1.hi, a2.hi, a3.hi, b0, b1);
-            }
-        }
-    }
-#pragma unroll
-    for (int c = 0; c < NCH; ++c)
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-            part[warp][c][q][lane] = acc[c][q];
-    __syncthreads();
-
     // accumulator q of lane (g,tq), chunk c: row g + 8*(q>>1), token c*8 + 2*tq + (q&1)
     for (int o = threadIdx.x; o < 16 * 8 * NCH; o += RL_WARPS * 32) {
         const int r = o & 15, slot = o >> 4;
@@ -157,6 +87,106 @@ router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restric
     }
 }
 
+// RB: blocks of 16 router rows per CTA.  With many experts and many tokens the kernel is bound by
+// what its CTAs re-read from L2 (every token tile once per row block, every row block once per
+// token tile); two row blocks per CTA share the token loads and halve the first term.
+template <int NCH, int RB>
+__global__ void __launch_bounds__(RL_WARPS_FOR(NCH) * 32)
+router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ w_router,
+                     const float *__restrict__ bias, const __nv_bfloat16 *__restrict__ w_sg,
+                     int T, int H, int E, int n_rows, float *__restrict__ logits,
+                     float *__restrict__ shared_scale, int32_t *__restrict__ zero, int zero_n)
+{
+    constexpr int RL_WARPS = RL_WARPS_FOR(NCH);
+    __shared__ float part[RL_WARPS][NCH][4][32];
+    griddep_wait();    // first kernel of a layer call: everything older is complete from here on
+    if (zero != nullptr && blockIdx.x == 0 && blockIdx.y == 0) {
+        // counters that a later kernel of this call updates before the plan kernel has run
+        for (int i = threadIdx.x; i < zero_n; i += blockDim.x)
+            zero[i] = 0;
+        __threadfence();
+        __syncthreads();
+    }
+    griddep_launch();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;
+    const int e0 = blockIdx.x * 16 * RB;
+    const int t0 = blockIdx.y * (8 * NCH);
+
+    auto row_src = [&](int e) {
+        RowSrc r{nullptr, nullptr};
+        if (e < E)
+            r.f32 = w_router + (size_t)e * H + 8 * tq;
+        else if (e == E && e < n_rows)
+            r.bf16 = w_sg + 8 * tq;
+        return r;
+    };
+    RowSrc rlo[RB], rhi[RB];
+#pragma unroll
+    for (int rb = 0; rb < RB; ++rb) {
+        rlo[rb] = row_src(e0 + 16 * rb + g);
+        rhi[rb] = row_src(e0 + 16 * rb + g + 8);
+    }
+    const __nv_bfloat16 *b[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c)
+        b[c] = x + (size_t)min(t0 + c * 8 + g, T - 1) * H + 8 * tq;
+
+    float acc[RB][NCH][4];
+#pragma unroll
+    for (int rb = 0; rb < RB; ++rb)
+#pragma unroll
+        for (int c = 0; c < NCH; ++c)
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                acc[rb][c][q] = 0.f;
+
+    const int nsteps = H >> 5;
+    const int s0 = warp * nsteps / RL_WARPS, s1 = (warp + 1) * nsteps / RL_WARPS;
+#pragma unroll 4
+    for (int s = s0; s < s1; ++s) {
+        const int k = s * 32;
+        uint4 B[NCH];
+#pragma unroll
+        for (int c = 0; c < NCH; ++c)
+            B[c] = ld_cached_v4(b[c] + k);
+#pragma unroll
+        for (int rb = 0; rb < RB; ++rb) {
+            float lo8[8], hi8[8];
+            load_row8(rlo[rb], k, lo8);
+            load_row8(rhi[rb], k, hi8);
+            // physical k positions 8tq+{0..3} feed the first MMA, 8tq+{4..7} the second
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const Split3 a0 = split_pair(lo8[4 * half + 0], lo8[4 * half + 1]);
+                const Split3 a1 = split_pair(hi8[4 * half + 0], hi8[4 * half + 1]);
+                const Split3 a2 = split_pair(lo8[4 * half + 2], lo8[4 * half + 3]);
+                const Split3 a3 = split_pair(hi8[4 * half + 2], hi8[4 * half + 3]);
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    const uint32_t b0 = half ? B[c].z : B[c].x, b1 = half ? B[c].w : B[c].y;
+                    mma_bf16_16816(acc[rb][c], a0.lo, a1.lo, a2.lo, a3.lo, b0, b1);
+                    mma_bf16_16816(acc[rb][c], a0.mid, a1.mid, a2.mid, a3.mid, b0, b1);
+                    mma_bf16_16816(acc[rb][c], a0.hi, a1.hi, a2.hi, a3.hi, b0, b1);
+                }
+            }
+        }
+    }
+
+#pragma unroll
+    for (int rb = 0; rb < RB; ++rb) {
+        if (rb > 0)
+            __syncthreads();  // the previous row block's sums have been read
+#pragma unroll
+        for (int c = 0; c < NCH; ++c)
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                part[warp][c][q][lane] = acc[rb][c][q];
+        __syncthreads();
+        reduce_and_store<NCH>(part, e0 + 16 * rb, t0, T, E, n_rows, bias, logits, shared_scale);
+    }
+}
+
 cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
                                  const __nv_bfloat16 *x, int T, float *logits,
                                  float *shared_scale, cudaStream_t s, int32_t *zero, int zero_n)
@@ -168,18 +198,26 @@ cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
     int nch = 1;
     while (nch < 8 && (long long)e_tiles * ((T + 8 * nch - 1) / (8 * nch)) > (long long)sm_count())
         nch *= 2;
-    dim3 grid(e_tiles, (T + 8 * nch - 1) / (8 * nch));
+    // two row blocks per CTA once the grid exceeds a wave of the largest token tile
+    const int token_tiles = (T + 8 * nch - 1) / (8 * nch);
+    const int rb = (nch == 8 && e_tiles >= 8 && (long long)e_tiles * token_tiles > (long long)sm_count()) ? 2 : 1;
+    dim3 grid((e_tiles + rb - 1) / rb, token_tiles);
     const __nv_bfloat16 *w_sg = static_cast<const __nv_bfloat16 *>(w.w_shared_gate);
-#define MOE_RL_LAUNCH(N)                                                                    \
-    err = launch_pdl(router_logits_kernel<N>, grid, dim3(RL_WARPS_FOR(N) * 32), 0, s, x, w.w_router,    \
+#define MOE_RL_LAUNCH(N, R)                                                                 \
+    err = launch_pdl(router_logits_kernel<N, R>, grid, dim3(RL_WARPS_FOR(N) * 32), 0, s, x, w.w_router, \
                      w.router_bias, w_sg, T, c.hidden, c.n_experts, n_rows, logits, shared_scale, zero,  \
                      zero_n)
     cudaError_t err = cudaSuccess;
     switch (nch) {
-    case 1: MOE_RL_LAUNCH(1); break;
-    case 2: MOE_RL_LAUNCH(2); break;
-    case 4: MOE_RL_LAUNCH(4); break;
-    default: MOE_RL_LAUNCH(8); break;
+    case 1: MOE_RL_LAUNCH(1, 1); break;
+    case 2: MOE_RL_LAUNCH(2, 1); break;
+    case 4: MOE_RL_LAUNCH(4, 1); break;
+    default:
+        if (rb == 2)
+            MOE_RL_LAUNCH(8, 2);
+        else
+            MOE_RL_LAUNCH(8, 1);
+        break;
     }
 #undef MOE_RL_LAUNCH
     return err;
