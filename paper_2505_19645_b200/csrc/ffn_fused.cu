@@ -1109,35 +1109,33 @@ cudaError_t launch_wait_limit_selftest(int32_t *status, int32_t *never_set, int 
 
 constexpr int GATHER_UNROLL = 8;
 
+// One warp per sorted row: the source token is looked up once per row (all lanes read the same
+// word), then the row is copied in passes of GATHER_UNROLL x 512 bytes whose loads are all in
+// flight before the first store.
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__restrict__ perm, int A,
                    int H, int top_k, __nv_bfloat16 *__restrict__ x_sorted)
 {
     griddep_launch();
     griddep_wait();
+    const int lane = threadIdx.x & 31;
+    const int warps = (int)((gridDim.x * blockDim.x) >> 5);
     const int vec_per_row = H >> 3;
-    const size_t total = (size_t)A * vec_per_row;
-    const size_t stride = (size_t)gridDim.x * blockDim.x;
-    // GATHER_UNROLL independent row pieces per thread and pass
-    for (size_t i0 = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i0 < total;
-         i0 += GATHER_UNROLL * stride) {
-        int r[GATHER_UNROLL], v[GATHER_UNROLL], t[GATHER_UNROLL];
-        uint4 d[GATHER_UNROLL];
+    for (int r = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5); r < A; r += warps) {
+        const int t = perm[r] / top_k;
+        const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)t * H);
+        uint4 *dst = reinterpret_cast<uint4 *>(x_sorted + (size_t)r * H);
+        for (int v0 = lane; v0 < vec_per_row; v0 += 32 * GATHER_UNROLL) {
+            uint4 d[GATHER_UNROLL];
 #pragma unroll
-        for (int u = 0; u < GATHER_UNROLL; ++u) {
-            const size_t i = i0 + u * stride;
-            r[u] = i < total ? (int)(i / vec_per_row) : -1;
-            v[u] = i < total ? (int)(i - (size_t)r[u] * vec_per_row) : 0;
-            t[u] = r[u] >= 0 ? perm[r[u]] / top_k : 0;
+            for (int u = 0; u < GATHER_UNROLL; ++u)
+                if (v0 + 32 * u < vec_per_row)
+                    d[u] = src[v0 + 32 * u];
+#pragma unroll
+            for (int u = 0; u < GATHER_UNROLL; ++u)
+                if (v0 + 32 * u < vec_per_row)
+                    dst[v0 + 32 * u] = d[u];
         }
-#pragma unroll
-        for (int u = 0; u < GATHER_UNROLL; ++u)
-            if (r[u] >= 0)
-                d[u] = reinterpret_cast<const uint4 *>(x + (size_t)t[u] * H)[v[u]];
-#pragma unroll
-        for (int u = 0; u < GATHER_UNROLL; ++u)
-            if (r[u] >= 0)
-                reinterpret_cast<uint4 *>(x_sorted + (size_t)r[u] * H)[v[u]] = d[u];
     }
 }
 
@@ -1151,9 +1149,8 @@ cudaError_t launch_gather_rows(const moe_config_t &c, const __nv_bfloat16 *x, co
     // finished the gate/up pass runs its shared-expert tiles only on the SMs this kernel
     // leaves alone.  Up to 16 MB of rows the gather therefore runs as one CTA per SM at most
     // (the hardware places them on about half of the SMs; fewer, larger CTAs made the gather
-    // itself too slow); a large gather needs every SM's full thread count to hide the two
-    // dependent loads of every row piece.
-    size_t blocks = (total + 255) / 256;
+    // itself too slow); a large gather needs every SM's full thread count.
+    size_t blocks = ((size_t)A + 7) / 8;  // a row per warp, eight warps per CTA
     const size_t cap = (size_t)sm_count() * (total * 16 <= (16u << 20) ? 1 : 8);
     if (blocks > cap)
         blocks = cap;
