@@ -146,7 +146,7 @@ moe_status_t moe_grouped_swiglu(const moe_config_t *cfg, const moe_weights_t *w,
  * until the process exits.  The call itself allocates nothing, on host or device.
  *
  * Limit: the request must satisfy, with A = T*top_k and every term rounded up to 256 bytes,
- *   256 + 64 + 52*(n_experts + A/128 + 1) + 4*(T/128 + 1) + 2*A*hidden + 2*A*inter + 2*T*shared_inter
+ *   256 + 64 + 52*(n_experts + A/128 + 1) + 4*(T/64 + 1) + 2*A*hidden + 2*A*inter + 2*T*shared_inter
  *     <= MOE_STATIC_SCRATCH_BYTES,
  * otherwise MOE_ERR_WORKSPACE is returned and nothing is launched (use moe_grouped_swiglu).
  *

@@ -48,7 +48,8 @@ struct PlanView {
     int32_t *done_shared;
 };
 
-__host__ __device__ inline int max_shared_segments(int T) { return (T + SEG_TOKENS - 1) / SEG_TOKENS; }
+// (the shared expert's rows may be cut into half segments, see the FFN launchers)
+__host__ __device__ inline int max_shared_segments(int T) { return (T + SEG_TOKENS / 2 - 1) / (SEG_TOKENS / 2); }
 
 __host__ __device__ inline int max_segments(int E, int A) { return E + A / SEG_TOKENS + 1; }
 

@@ -98,6 +98,10 @@ struct FfnArgs {
     int n_w_slots;
     int x_units;       // token ring size in FF_X_UNIT units
     int wait_us;       // limit of every wait inside the kernel, microseconds
+    int shared_seg;    // token rows per segment of the shared expert: FF_SEG, or half of it
+                       // for 64 < T <= 128, where two 64-row segments are run as single items so
+                       // that no token entry exceeds 16 KB and the ring can be small
+    int shared_paired; // two segments of the shared expert share one pass over a tile
 };
 
 // Tensor maps of one pass: weights [kind][matrix][box height], token operand [kind][box height].
@@ -373,7 +377,7 @@ struct ItemWalk {
     Segment sg;
     int g_nseg, g_u_end;
     bool have_tile;
-    int t_grp, t_expert, t_u0, t_h, t_row0, t_n, t_s, t_s_end, t_seg0;
+    int t_grp, t_expert, t_u0, t_h, t_row0, t_n, t_s, t_s_end, t_seg0, t_s0, t_seg_rows;
     bool t_once;  // the tile's weights are read by this pass over it only
     int t_k0, t_k1;
     long long t_out_off;
@@ -390,8 +394,8 @@ struct ItemWalk {
         s_base = a.shared_tiles ? Us / a.shared_tiles : 0;
         s_rem = a.shared_tiles ? Us % a.shared_tiles : 0;
         sj = blockIdx.x;
-        nseg_s = (a.T + FF_SEG - 1) / FF_SEG;
-        pairs_s = (nseg_s + 1) >> 1;
+        nseg_s = (a.T + a.shared_seg - 1) / a.shared_seg;
+        pairs_s = a.shared_paired ? (nseg_s + 1) >> 1 : nseg_s;
         s_units = a.shared_tiles * a.shared_ksplit * pairs_s;
         R0 = a.rows[0] >> 4;
         nseg_total = fs = u = fs_hi = u_hi = 0;
@@ -528,10 +532,10 @@ struct ItemWalk {
                     it.expert = t_expert;
                     it.f0 = t_u0 << 4;
                     it.h = t_h << 4;
-                    it.row0 = t_row0 + t_s * FF_SEG;
-                    it.n = min(FF_SEG, t_n - t_s * FF_SEG);
-                    // segments 2q and 2q+1 of a tile form a pair
-                    it.role = (t_s & 1) ? 2 : (t_s + 1 < t_s_end ? 1 : 0);
+                    it.row0 = t_row0 + t_s * t_seg_rows;
+                    it.n = min(t_seg_rows, t_n - t_s * t_seg_rows);
+                    // the segments of a tile pair up from its first one on
+                    it.role = ((t_s - t_s0) & 1) ? 2 : (t_s + 1 < t_s_end ? 1 : 0);
                     it.seg = t_seg0 + t_s;
                     it.w_once = t_once;
                     it.k0 = t_k0;
@@ -555,9 +559,11 @@ struct ItemWalk {
                 t_row0 = 0;
                 t_seg0 = 0;
                 t_n = a.T;
-                t_s = 2 * q;
-                t_s_end = min(nseg_s, 2 * q + 2);
-                t_once = nseg_s <= 2;
+                t_seg_rows = a.shared_seg;
+                t_s = a.shared_paired ? 2 * q : q;
+                t_s0 = t_s;
+                t_s_end = a.shared_paired ? min(nseg_s, 2 * q + 2) : q + 1;
+                t_once = pairs_s <= 1;
                 sj += gridDim.x;
                 have_tile = true;
                 continue;
@@ -584,7 +590,9 @@ struct ItemWalk {
                     t_row0 = sg.row0;
                     t_seg0 = sg.first_seg;
                     t_n = sg.n;
+                    t_seg_rows = FF_SEG;
                     t_s = sidx - sg.first_seg;
+                    t_s0 = t_s;
                     t_s_end = min(g_nseg, t_s + 2);
                     t_once = g_nseg <= 2;
                     t_k0 = chunk * a.routed_kchunk;
@@ -616,7 +624,9 @@ struct ItemWalk {
                 t_row0 = sg.row0;
                 t_seg0 = sg.first_seg;
                 t_n = sg.n;
+                t_seg_rows = FF_SEG;
                 t_s = 0;
+                t_s0 = 0;
                 t_s_end = g_nseg;
                 t_once = g_nseg <= 2;
                 t_k0 = 0;
@@ -1215,6 +1225,13 @@ static double expected_active_experts(int E, int k, int T)
 
 static int ffn_grid() { return sm_count(); }
 
+// Token rows per segment of the shared expert.  Up to 128 tokens no group of the layer has more
+// than one 128-row segment, so no two token entries must be resident together and the token
+// ring can be 32 KB, which leaves room for a third weight slot (worth 3-4 % of the layer) --
+// provided no entry exceeds half the ring: between 65 and 128 tokens the shared expert's rows
+// are therefore cut into two 64-row segments that run as single items.
+static int shared_segment_rows(int T) { return (T > FF_SEG / 2 && T <= FF_SEG) ? FF_SEG / 2 : FF_SEG; }
+
 // Number of tiles the shared expert's rows are cut into.  The shared expert's work units are
 // (tile, segment pair); a unit should cost about the expected per-CTA share of the whole pass
 // (or less), with the tile height within [min_tile, max_tile] rows: a tensor-core
@@ -1224,8 +1241,8 @@ static int shared_tile_count(const moe_config_t &c, int T, int rows_routed, int 
                              int K_routed, int K_shared, int ksplit, int min_tile, int max_tile,
                              int grid)
 {
-    const int nseg_s = (T + FF_SEG - 1) / FF_SEG;
-    const int pairs_s = (nseg_s + 1) / 2;
+    const int nseg_s = (T + shared_segment_rows(T) - 1) / shared_segment_rows(T);
+    const int pairs_s = T > FF_SEG ? (nseg_s + 1) / 2 : nseg_s;
     const int units = rows_shared >> 4;
     const double k_ratio = (double)K_shared / K_routed;  // cost of a shared row unit per segment
     const double n_act = expected_active_experts(c.n_experts, c.top_k, T);
@@ -1248,12 +1265,12 @@ static void ffn_geometry(int T, FfnArgs &a)
     const char *ekb = getenv("MOE_FF_KBOXES"), *exr = getenv("MOE_FF_XRING_KB");
     a.kboxes = ekb ? atoi(ekb) : 2;
     a.w_slot_bytes = 256 * 128 * a.kboxes;  // a full tile: 256 stacked rows per k box
-    int x_ring_bytes = T > 64 ? 96 * 1024 : 32 * 1024;
+    int x_ring_bytes = T > FF_SEG ? 96 * 1024 : 32 * 1024;
     if (exr)
         x_ring_bytes = atoi(exr) * 1024;
     // entries never wrap, so two entries that must be resident together (a pair of segments:
     // 32 KB + up to 32 KB) need a ring of three of them wherever the first may sit
-    if (T > 64 && x_ring_bytes < 96 * 1024)
+    if (T > FF_SEG && x_ring_bytes < 96 * 1024)
         x_ring_bytes = 96 * 1024;
     if (x_ring_bytes < 32 * 1024)
         x_ring_bytes = 32 * 1024;
@@ -1264,6 +1281,8 @@ static void ffn_geometry(int T, FfnArgs &a)
         ns = FF_MAX_W_SLOTS;
     a.n_w_slots = ns;
     a.wait_us = (int)(FF_WAIT_NS / 1000ull);
+    a.shared_seg = shared_segment_rows(T);
+    a.shared_paired = T > FF_SEG ? 1 : 0;
 }
 
 // Range mode keeps every CTA alone on "its" groups, perfectly levelled.  It loses when

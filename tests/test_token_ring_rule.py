@@ -5,7 +5,7 @@ entry that does not fit before the end of the ring starts at unit 0, and the pro
 entry j once everything before the oldest entry still in use is free.  The MMA side consumes
 the entries of one k step together (one entry, or two for a pair of segments).  This test
 replays that rule over random item sequences: the geometries the host chooses (48 units with
-pairs of segments, 16 units without) never stall and never overlap live entries, and a ring
+pairs of segments, 16 units without, i.e. up to 128 tokens) never stall and never overlap live entries, and a ring
 of exactly two full entries with pairs does stall -- which is why the host refuses it.
 """
 import random
@@ -88,9 +88,14 @@ def test_ring_of_three_full_entries_never_stalls_with_pairs():
 
 
 def test_small_ring_never_stalls_without_pairs():
+    """Up to 128 tokens no group has two segments: single entries only, of up to half the ring
+    (the shared expert's 64-row segments, groups of up to 64 rows) or, for a routed group of up
+    to 128 rows, of the whole ring."""
     rng = random.Random(2)
     for _ in range(4000):
         assert replay(16, random_steps(rng, 4, False)) == "ok"
+    for _ in range(4000):
+        assert replay(16, random_steps(rng, 8, False)) == "ok"
 
 
 def test_ring_of_two_full_entries_can_stall_with_pairs():
