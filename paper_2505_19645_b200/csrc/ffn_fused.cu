@@ -1225,12 +1225,28 @@ static double expected_active_experts(int E, int k, int T)
 
 static int ffn_grid() { return sm_count(); }
 
-// Token rows per segment of the shared expert.  Up to 128 tokens no group of the layer has more
-// than one 128-row segment, so no two token entries must be resident together and the token
-// ring can be 32 KB, which leaves room for a third weight slot (worth 3-4 % of the layer) --
-// provided no entry exceeds half the ring: between 65 and 128 tokens the shared expert's rows
-// are therefore cut into two 64-row segments that run as single items.
-static int shared_segment_rows(int T) { return (T > FF_SEG / 2 && T <= FF_SEG) ? FF_SEG / 2 : FF_SEG; }
+// Up to 128 tokens no group of the layer has more than one 128-row segment, so no two token
+// entries must be resident together and the token ring can be 32 KB, which leaves room for a
+// third weight slot (worth 3-4 % of the layer) -- provided the entries stay within half of the
+// ring, i.e. 64 rows: always so up to 64 tokens; between 65 and 128 tokens only while the
+// routed groups are expected to be small (a larger group still works, its rows are then not
+// fetched ahead), and the shared expert's rows are then cut into two 64-row segments that run
+// as single items.
+static bool small_token_ring(const moe_config_t &c, int T)
+{
+    if (T <= FF_SEG / 2)
+        return true;
+    if (T > FF_SEG)
+        return false;
+    // (a mean of up to a quarter of a segment: the largest group then stays within a half)
+    return (double)T * c.top_k / expected_active_experts(c.n_experts, c.top_k, T) <= FF_SEG / 4 + 0.5;
+}
+
+// Token rows per segment of the shared expert (see small_token_ring).
+static int shared_segment_rows(const moe_config_t &c, int T)
+{
+    return (T > FF_SEG / 2 && small_token_ring(c, T)) ? FF_SEG / 2 : FF_SEG;
+}
 
 // Number of tiles the shared expert's rows are cut into.  The shared expert's work units are
 // (tile, segment pair); a unit should cost about the expected per-CTA share of the whole pass
@@ -1241,7 +1257,7 @@ static int shared_tile_count(const moe_config_t &c, int T, int rows_routed, int 
                              int K_routed, int K_shared, int ksplit, int min_tile, int max_tile,
                              int grid)
 {
-    const int nseg_s = (T + shared_segment_rows(T) - 1) / shared_segment_rows(T);
+    const int nseg_s = (T + shared_segment_rows(c, T) - 1) / shared_segment_rows(c, T);
     const int pairs_s = T > FF_SEG ? (nseg_s + 1) / 2 : nseg_s;
     const int units = rows_shared >> 4;
     const double k_ratio = (double)K_shared / K_routed;  // cost of a shared row unit per segment
@@ -1260,12 +1276,12 @@ static int shared_tile_count(const moe_config_t &c, int T, int rows_routed, int 
 // 256 contiguous bytes, which both HBM and L2 serve markedly faster than 128).  The token
 // ring holds two entries of the largest possible segment while no group can exceed 64 rows,
 // three 128-row entries otherwise (a pair of segments needs two at once).
-static void ffn_geometry(int T, FfnArgs &a)
+static void ffn_geometry(const moe_config_t &c, int T, FfnArgs &a)
 {
     const char *ekb = getenv("MOE_FF_KBOXES"), *exr = getenv("MOE_FF_XRING_KB");
     a.kboxes = ekb ? atoi(ekb) : 2;
     a.w_slot_bytes = 256 * 128 * a.kboxes;  // a full tile: 256 stacked rows per k box
-    int x_ring_bytes = T > FF_SEG ? 96 * 1024 : 32 * 1024;
+    int x_ring_bytes = small_token_ring(c, T) ? 32 * 1024 : 96 * 1024;
     if (exr)
         x_ring_bytes = atoi(exr) * 1024;
     // entries never wrap, so two entries that must be resident together (a pair of segments:
@@ -1281,7 +1297,7 @@ static void ffn_geometry(int T, FfnArgs &a)
         ns = FF_MAX_W_SLOTS;
     a.n_w_slots = ns;
     a.wait_us = (int)(FF_WAIT_NS / 1000ull);
-    a.shared_seg = shared_segment_rows(T);
+    a.shared_seg = shared_segment_rows(c, T);
     a.shared_paired = T > FF_SEG ? 1 : 0;
 }
 
@@ -1343,7 +1359,7 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
     a.shared_tiles = with_shared ? shared_tile_count(c, T, c.inter, c.shared_inter, c.hidden, c.hidden,
                                                      1, 64, 128, ffn_grid())
                                  : 0;
-    ffn_geometry(T, a);
+    ffn_geometry(c, T, a);
     FfnMaps maps;
     memset(&maps, 0, sizeof maps);
     bool ok = make_weight_maps(maps.w[0][0], w.w_gate, E * c.inter, H) &&
@@ -1455,7 +1471,7 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
     a.shared_tiles = with_shared ? shared_tile_count(c, T, c.hidden, c.hidden, c.inter, c.shared_inter,
                                                      a.shared_ksplit, 128, 256, ffn_grid())
                                  : 0;
-    ffn_geometry(T, a);
+    ffn_geometry(c, T, a);
     FfnMaps maps;
     memset(&maps, 0, sizeof maps);
     bool ok = make_weight_maps(maps.w[0][0], w.w_down, E * H, c.inter) &&
