@@ -34,7 +34,7 @@ DEFAULT_CONFIG = "qwen1.5-moe-a2.7b"
 DEFAULT_B, DEFAULT_GAMMA = 32, 3
 # dram__bytes_read.sum + dram__bytes_write.sum of one gate/up launch on the default workload
 # (profiles/ffn_fused_qwen15_T128.md); set to None whenever that kernel changes
-NCU_GATE_UP_DRAM_BYTES = 740941568 + 5508864
+NCU_GATE_UP_DRAM_BYTES = 741085440 + 3427840
 
 
 def load_peaks():
