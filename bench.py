@@ -416,13 +416,13 @@ def main():
     sweep = []
     if not args.no_sweep and rank == 0:
         Bs, gs = sweep_grid(args)
-        # Two passes over the grid, half of the samples in each.  A point takes tens of
+        # Three passes over the grid, a third of the samples in each.  A point takes tens of
         # milliseconds and the part's clock steps on that time scale at its power cap, so a
-        # single visit can fall into a slow step as a whole; the lower of the two medians
-        # counts and both are recorded.
+        # single visit can fall into a slow step as a whole; the lowest of the three medians
+        # counts and all are recorded.
         rounds = {}
-        per_round = max(5, args.sweep_steps // 2)
-        for _ in range(2):
+        per_round = max(5, args.sweep_steps // 3)
+        for _ in range(3):
             for Bi in Bs:
                 for gi in gs:
                     Ti = Bi * (gi + 1)
