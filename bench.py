@@ -420,23 +420,23 @@ def main():
         # milliseconds and the part's clock steps on that time scale at its power cap, so a
         # single visit can fall into a slow step as a whole; the lowest of the three medians
         # counts and all are recorded.
-        rounds = {}
-        per_round = max(5, args.sweep_steps // 3)
+        passes = {}
+        per_pass = max(5, args.sweep_steps // 3)
         for _ in range(3):
             for Bi in Bs:
                 for gi in gs:
                     Ti = Bi * (gi + 1)
                     xi = wl.make_tokens(shape, Ti, wl.point_seed(args.config, Bi, gi), device)
-                    ms, _ = runner.time_steps(xi, Bi, gi, per_round, 3)
-                    rounds.setdefault((Bi, gi), []).append(ms)
+                    ms, _ = runner.time_steps(xi, Bi, gi, per_pass, 3)
+                    passes.setdefault((Bi, gi), []).append(ms)
         for Bi in Bs:
             base_ms = None
             for gi in gs:
                 Ti = Bi * (gi + 1)
                 xi = wl.make_tokens(shape, Ti, wl.point_seed(args.config, Bi, gi), device)
                 na = runner.n_active(xi, Bi, gi)
-                medians = [statistics.median(r) for r in rounds[(Bi, gi)]]
-                ms = [v for r in rounds[(Bi, gi)] for v in r]
+                medians = [statistics.median(r) for r in passes[(Bi, gi)]]
+                ms = [v for r in passes[(Bi, gi)] for v in r]
                 med = min(medians)
                 if gi == gs[0]:
                     base_ms = med
