@@ -6,9 +6,14 @@
 // values are exact, and the three partial products are accumulated in fp32 by
 // m16n8k16 MMAs.  A CTA owns 16 router rows x (8*NCH) tokens; its 16 warps split H and are
 // summed through shared memory, so even T = 1 keeps every load short and parallel.
+#include <cooperative_groups.h>
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace moe {
+
+namespace cg = cooperative_groups;
 
 // warps per CTA (they split H): 16 for the small token tiles that latency-bound calls use
 #define RL_WARPS_FOR(nch) ((nch) <= 2 ? 16 : 8)
@@ -87,6 +92,48 @@ __device__ __forceinline__ void reduce_and_store(const float (&part)[RL_WARPS_FO
     }
 }
 
+// The same for a cluster of CTAs that split H between them (few tokens, few row blocks: one CTA
+// per row block would leave most SMs idle and each CTA a long reduction).  Every CTA sums its
+// warps into `red`; the cluster's first CTA adds the CTAs' sums in rank order through
+// distributed shared memory -- a fixed order, so the logits do not depend on timing.
+template <int NCH>
+__device__ __forceinline__ void reduce_cluster_and_store(
+    const float (&part)[RL_WARPS_FOR(NCH)][NCH][4][32], float (&red)[16 * 8 * NCH], int e0, int t0,
+    int T, int E, int n_rows, const float *__restrict__ bias, float *__restrict__ logits,
+    float *__restrict__ shared_scale)
+{
+    constexpr int RL_WARPS = RL_WARPS_FOR(NCH);
+    cg::cluster_group cluster = cg::this_cluster();
+    for (int o = threadIdx.x; o < 16 * 8 * NCH; o += RL_WARPS * 32) {
+        const int r = o & 15, slot = o >> 4;
+        const int c = slot >> 3, tt = (slot & 7) >> 1, lo = slot & 1;
+        const int q = ((r >> 3) << 1) | lo, ln = ((r & 7) << 2) | tt;
+        float v = 0.f;
+#pragma unroll
+        for (int w = 0; w < RL_WARPS; ++w)
+            v += part[w][c][q][ln];
+        red[o] = v;
+    }
+    cluster.sync();
+    if (cluster.block_rank() == 0) {
+        const unsigned n = cluster.num_blocks();
+        for (int o = threadIdx.x; o < 16 * 8 * NCH; o += RL_WARPS * 32) {
+            const int r = o & 15, slot = o >> 4;
+            const int e = e0 + r, t = t0 + slot;
+            if (e >= n_rows || t >= T)
+                continue;
+            float v = red[o];
+            for (unsigned k = 1; k < n; ++k)
+                v += cluster.map_shared_rank(&red[0], k)[o];
+            if (e < E)
+                logits[(size_t)t * E + e] = bias ? v + bias[e] : v;
+            else
+                shared_scale[t] = 1.0f / (1.0f + expf(-v));
+        }
+    }
+    cluster.sync();  // the other CTAs' shared memory stays valid until it has been read
+}
+
 // RB: blocks of 16 router rows per CTA.  With many experts and many tokens the kernel is bound by
 // what its CTAs re-read from L2 (every token tile once per row block, every row block once per
 // token tile); two row blocks per CTA share the token loads and halve the first term.
@@ -141,8 +188,11 @@ router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restric
             for (int q = 0; q < 4; ++q)
                 acc[rb][c][q] = 0.f;
 
-    const int nsteps = H >> 5;
-    const int s0 = warp * nsteps / RL_WARPS, s1 = (warp + 1) * nsteps / RL_WARPS;
+    // gridDim.z CTAs (one cluster) split H; the warps of a CTA split the CTA's share
+    const int nsteps_all = H >> 5;
+    const int z0 = blockIdx.z * nsteps_all / gridDim.z, z1 = (blockIdx.z + 1) * nsteps_all / gridDim.z;
+    const int nsteps = z1 - z0;
+    const int s0 = z0 + warp * nsteps / RL_WARPS, s1 = z0 + (warp + 1) * nsteps / RL_WARPS;
 #pragma unroll 4
     for (int s = s0; s < s1; ++s) {
         const int k = s * 32;
@@ -183,6 +233,14 @@ router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restric
             for (int q = 0; q < 4; ++q)
                 part[warp][c][q][lane] = acc[rb][c][q];
         __syncthreads();
+        if constexpr (RB == 1 && NCH == 1) {
+            if (gridDim.z > 1) {
+                __shared__ float red[16 * 8 * NCH];
+                reduce_cluster_and_store<NCH>(part, red, e0, t0, T, E, n_rows, bias, logits,
+                                              shared_scale);
+                continue;
+            }
+        }
         reduce_and_store<NCH>(part, e0 + 16 * rb, t0, T, E, n_rows, bias, logits, shared_scale);
     }
 }
@@ -202,6 +260,44 @@ cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
     const int token_tiles = (T + 8 * nch - 1) / (8 * nch);
     const int rb = (nch == 8 && e_tiles >= 8 && (long long)e_tiles * token_tiles > (long long)sm_count()) ? 2 : 1;
     dim3 grid((e_tiles + rb - 1) / rb, token_tiles);
+    // Few row blocks and few tokens with a long reduction (eight and more 32-element steps per
+    // warp: below that the cluster launch costs what the shorter loops save): clusters of up
+    // to eight CTAs split H, as long as the grid stays within one wave and every warp keeps at
+    // least one step.
+    int ks = 1;
+    if (nch == 1 && (c.hidden >> 5) / RL_WARPS_FOR(1) >= 8) {
+        static const bool split = [] {
+            const char *e = getenv("MOE_RL_KSPLIT");
+            return !e || atoi(e) != 0;
+        }();
+        ks = split ? 8 : 1;
+        while (ks > 1 && ((long long)e_tiles * token_tiles * ks > (long long)sm_count() ||
+                          (c.hidden >> 5) / ks < RL_WARPS_FOR(1)))
+            ks /= 2;
+    }
+    if (ks > 1) {
+        grid.z = ks;
+        void (*kernel)(const __nv_bfloat16 *, const float *, const float *, const __nv_bfloat16 *, int,
+                       int, int, int, float *, float *, int32_t *, int) = router_logits_kernel<1, 1>;
+        prefer_max_shared_carveout(reinterpret_cast<const void *>(kernel));
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = grid;
+        cfg.blockDim = dim3(RL_WARPS_FOR(1) * 32);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = 1;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = ks;
+        cfg.attrs = attr;
+        cfg.numAttrs = 2;
+        return cudaLaunchKernelEx(&cfg, kernel, x, w.w_router, w.router_bias,
+                                  static_cast<const __nv_bfloat16 *>(w.w_shared_gate), T, c.hidden,
+                                  c.n_experts, n_rows, logits, shared_scale, zero, zero_n);
+    }
     const __nv_bfloat16 *w_sg = static_cast<const __nv_bfloat16 *>(w.w_shared_gate);
 #define MOE_RL_LAUNCH(N, R)                                                                 \
     err = launch_pdl(router_logits_kernel<N, R>, grid, dim3(RL_WARPS_FOR(N) * 32), 0, s, x, w.w_router, \
