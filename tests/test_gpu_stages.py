@@ -111,7 +111,10 @@ def test_permute_bit_exact(T, k, E, mode):
                                              (130, 7168, 256, True, False), (9, 96, 3, True, True),
                                              # two row blocks per CTA: many experts x many tokens,
                                              # an odd number of row blocks, a ragged token tile
-                                             (700, 512, 256, True, False), (1000, 256, 200, False, True)])
+                                             (700, 512, 256, True, False), (1000, 256, 200, False, True),
+                                             # few tokens, long rows: clusters of CTAs split H
+                                             (1, 4096, 8, False, False), (5, 7168, 256, True, False),
+                                             (16, 4096, 60, False, True), (3, 4128, 17, True, True)])
 def test_router_logits(T, H, E, bias, gate):
     api = _api()
     shape = wl.small_shape("l", H, E, 1, 64, 64 if gate else 0, 0, 0, 1 if gate else 0)
