@@ -88,8 +88,17 @@ typedef struct {
     int32_t *n_active; /* [1]      */
 } moe_debug_out_t;
 
-/* Bytes of workspace any entry point needs for up to max_tokens tokens (0 on bad args). */
+/* Bytes of workspace any entry point needs for up to max_tokens tokens (0 on bad args).
+ * The workspace need not be initialised. */
 size_t moe_workspace_bytes(const moe_config_t *cfg, int32_t max_tokens);
+
+/* Test aid (no counterpart in the paper): region `index` (0, 1, ...) of the layout a call with T
+ * tokens uses inside its workspace, as byte offset and bytes in use.  Regions start 256-byte
+ * aligned and are separated by at least 256 bytes that no kernel ever writes, so a caller that
+ * fills the workspace with a pattern first can detect a stray store afterwards.  Returns
+ * MOE_ERR_INVALID_ARG past the last region. */
+moe_status_t moe_workspace_region(const moe_config_t *cfg, int32_t T, int32_t index,
+                                  size_t *offset, size_t *bytes);
 
 /* Router logits (the gate of Sec. 1):  logits[t,e] = x[t,:] . w_router[e,:] (+ bias[e]),
  * fp32 accumulation.  If shared_scale != NULL and cfg->shared_gate, also writes
@@ -145,7 +154,8 @@ moe_status_t moe_grouped_swiglu(const moe_config_t *cfg, const moe_weights_t *w,
  * MOE_STATIC_SCRATCH_BYTES inside the library image; each GPU that loads the library holds it
  * until the process exits.  The call itself allocates nothing, on host or device.
  *
- * Limit: the request must satisfy, with A = T*top_k and every term rounded up to 256 bytes,
+ * Limit: the request must satisfy, with A = T*top_k and every term rounded up to 256 bytes and
+ * followed by 256 bytes of guard,
  *   256 + 64 + 52*(n_experts + A/128 + 1) + 4*(T/64 + 1) + 2*A*hidden + 2*A*inter + 2*T*shared_inter
  *     <= MOE_STATIC_SCRATCH_BYTES,
  * otherwise MOE_ERR_WORKSPACE is returned and nothing is launched (use moe_grouped_swiglu).
@@ -155,13 +165,27 @@ moe_status_t moe_grouped_swiglu(const moe_config_t *cfg, const moe_weights_t *w,
  * Sharing: every call on a device uses the same array and leaves its contents behind; the
  * call clears what it needs cleared.  Two calls whose work overlaps on the GPU (different
  * streams, or threads) race on it -- order them on one stream or with events.
- * Arguments, results and error codes otherwise as for moe_grouped_swiglu. */
+ * Arguments, results and host-side error codes otherwise as for moe_grouped_swiglu; the
+ * device-side status (a bounded wait that gave up) is read with moe_check_static. */
 #define MOE_STATIC_SCRATCH_BYTES (8u << 20)
 moe_status_t moe_grouped_swiglu_static(const moe_config_t *cfg, const moe_weights_t *w,
                                        const void *x, int32_t T, const int32_t *offsets,
                                        const int32_t *perm, const int32_t *active,
                                        const int32_t *n_active, void *y, void *shared_y,
                                        void *stream);
+
+/* moe_check for moe_grouped_swiglu_static (no counterpart in the paper): synchronises `stream`
+ * and reports the status word inside the library's scratch array of the current device --
+ * MOE_OK, MOE_ERR_TIMEOUT (a bounded wait inside a kernel of some static call since the last
+ * report gave up; that call's outputs are invalid, the context stays usable), or MOE_ERR_CUDA.
+ * The word is shared by every static call on the device and is cleared by this report.
+ * Allocates nothing. */
+moe_status_t moe_check_static(void *stream);
+
+/* moe_selftest_wait_limit on the status word of the library's scratch array: lets a caller of
+ * the static entry point see the failure path end to end (report through moe_check_static,
+ * next call unaffected) without anything faulting. */
+moe_status_t moe_selftest_wait_limit_static(int32_t limit_us, void *stream);
 
 /* Gate-weighted combine:
  *   out[t,:] = sum_{j<K} topk_w[t,j] * y[inv_perm[t*K+j],:]  (slot order, fp32)
@@ -177,14 +201,23 @@ moe_status_t moe_combine(const moe_config_t *cfg, const void *y, const int32_t *
  * moe_grouped_swiglu and moe_combine; the result equals the dense-masked definition
  *   out[t] = sum_e m[t,e] * FFN_e(x[t]) + s[t] * FFN_shared(x[t]).
  * T_T(B,gamma) of Sec. 3.1 is the duration of this call's work.
- *   x, out [T,H] bf16; dbg NULL or pointers that receive copies of the intermediates. */
+ *   x, out [T,H] bf16; dbg NULL or pointers that receive copies of the intermediates.
+ * Numerics: as the separate steps, except that while the down projection has too few work
+ * items to keep every SM streaming (few tokens, or few experts with long reductions) its
+ * reduction is cut into up to 8 k chunks whose partial sums are rounded to bf16 before the
+ * combine adds them in fp32: an expert output then carries up to 8 bf16 roundings instead of
+ * one, the shared expert's likewise (its chunk count depends on the shape only).  How many
+ * chunks are used depends on T, so a token's low-order bits may differ between batch sizes;
+ * the result stays within the layer's stated tolerance at every size. */
 moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, const void *x,
                               int32_t B, int32_t gamma, void *out, const moe_debug_out_t *dbg,
                               void *ws, size_t ws_bytes, void *stream);
 
 /* Synchronises `stream` and returns the device-side status word of the workspace:
  * MOE_OK, MOE_ERR_TIMEOUT if a bounded wait inside a kernel gave up (outputs are then
- * invalid but the context stays usable), or MOE_ERR_CUDA. */
+ * invalid but the context stays usable), or MOE_ERR_CUDA.  The word is sticky: a wait that
+ * gave up in ANY call on this workspace since the last report keeps it raised (later calls do
+ * not clear it), and this call clears it after reading, so every failure is reported once. */
 moe_status_t moe_check(void *ws, void *stream);
 
 /* Self-test of the failure path (no counterpart in the paper).  Every wait inside the kernels is

@@ -22,7 +22,8 @@ STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_UNSUPPORTED",
 EXPORTS = ["moe_workspace_bytes", "moe_router_logits", "moe_route_topk", "moe_permute",
            "moe_grouped_swiglu", "moe_combine", "moe_verify_layer", "moe_check",
            "moe_last_launch_count", "moe_status_string", "moe_profile_stage",
-           "moe_selftest_wait_limit"]
+           "moe_selftest_wait_limit", "moe_workspace_region", "moe_grouped_swiglu_static",
+           "moe_check_static", "moe_selftest_wait_limit_static"]
 
 STAGES = {"router_logits": 0, "route_topk": 1, "permute": 2, "plan": 3, "gate_up": 4, "down": 5,
           "combine": 6, "gather": 7}
@@ -91,6 +92,14 @@ def load_library():
     lib.moe_profile_stage.argtypes = [i32, vp, vp]
     lib.moe_selftest_wait_limit.restype = i32
     lib.moe_selftest_wait_limit.argtypes = [vp, i32, vp]
+    lib.moe_workspace_region.restype = i32
+    lib.moe_workspace_region.argtypes = [cfgp, i32, i32, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+    lib.moe_grouped_swiglu_static.restype = i32
+    lib.moe_grouped_swiglu_static.argtypes = [cfgp, wp, vp, i32] + [vp] * 7
+    lib.moe_check_static.restype = i32
+    lib.moe_check_static.argtypes = [vp]
+    lib.moe_selftest_wait_limit_static.restype = i32
+    lib.moe_selftest_wait_limit_static.argtypes = [i32, vp]
     lib.moe_last_launch_count.restype = i32
     lib.moe_last_launch_count.argtypes = []
     lib.moe_status_string.restype = ctypes.c_char_p
@@ -216,14 +225,34 @@ def moe_grouped_swiglu_static(cfg, weights, x, grouping: Grouping, y, shared_y, 
     g = grouping
     i32 = torch.int32
     lib = load_library()
-    lib.moe_grouped_swiglu_static.restype = ctypes.c_int32
-    lib.moe_grouped_swiglu_static.argtypes = [
-        ctypes.POINTER(CConfig), ctypes.POINTER(CWeights), ctypes.c_void_p, ctypes.c_int32] + \
-        [ctypes.c_void_p] * 7
     _check(lib.moe_grouped_swiglu_static(
         ctypes.byref(cfg), ctypes.byref(weights), _ptr(x, torch.bfloat16), T, _ptr(g.offsets, i32),
         _ptr(g.perm, i32), _ptr(g.active, i32), _ptr(g.n_active, i32), _ptr(y, torch.bfloat16),
         _ptr(shared_y, torch.bfloat16), _stream_ptr(stream)), "moe_grouped_swiglu_static")
+
+
+def moe_check_static(stream=None):
+    """moe_check for the static entry point: synchronises the stream and raises MoeError
+    (MOE_ERR_TIMEOUT) if a bounded wait gave up in a static call since the last report."""
+    _check(load_library().moe_check_static(_stream_ptr(stream)), "moe_check_static")
+
+
+def moe_selftest_wait_limit_static(limit_us: int, stream=None):
+    _check(load_library().moe_selftest_wait_limit_static(int(limit_us), _stream_ptr(stream)),
+           "moe_selftest_wait_limit_static")
+
+
+def workspace_regions(cfg: CConfig, T: int):
+    """[(offset, bytes)] of every region a call with T tokens uses inside its workspace."""
+    lib = load_library()
+    out = []
+    off, n = ctypes.c_size_t(), ctypes.c_size_t()
+    i = 0
+    while lib.moe_workspace_region(ctypes.byref(cfg), int(T), i, ctypes.byref(off),
+                                   ctypes.byref(n)) == MOE_OK:
+        out.append((int(off.value), int(n.value)))
+        i += 1
+    return out
 
 
 def moe_combine(cfg, y, inv_perm, topk_w, shared_y, shared_scale, out, stream=None):

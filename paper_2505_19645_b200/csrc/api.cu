@@ -53,6 +53,15 @@ bool pdl_enabled()
     return on;
 }
 
+int schedule_override()
+{
+    static const int v = [] {
+        const char *e = getenv("MOE_FF_RR");
+        return !e ? -1 : (e[0] == '1' ? 1 : (e[0] == '0' ? 0 : -1));
+    }();
+    return v;
+}
+
 static thread_local int g_last_launches = 0;
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -149,6 +158,19 @@ static thread_local bool g_probe_armed = false;  // only moe_verify_layer arms i
         if (probe_ && cudaEventRecord(g_probe.stop, s) != cudaSuccess)        \
             return MOE_ERR_CUDA;                                              \
     } while (0)
+
+// The stream must be idle.  A raised word is reported once: it is cleared after it has been read.
+moe_status_t read_and_clear_status(void *status_region)
+{
+    int32_t word[2] = {0, 0};
+    if (cudaMemcpy(word, status_region, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    if (word[1] != STATUS_MAGIC || word[0] == 0)
+        return MOE_OK;  // never initialised: no call has run on this workspace yet
+    if (cudaMemset(status_region, 0, sizeof(int32_t)) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    return MOE_ERR_TIMEOUT;
+}
 
 PlanView plan_view(char *ws, const Workspace &L)
 {
@@ -348,13 +370,13 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
         Arm() { g_probe_armed = true; }
         ~Arm() { g_probe_armed = false; }
     } arm;
-    MOE_STAGE(MOE_STAGE_ROUTER_LOGITS,
-              launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s,
-                                   plan_view(base, L).done_shared, max_shared_segments(T)));
-    // the grouping kernel also writes the FFN segment plan (one launch fewer); for a small
-    // batch it selects the experts and gathers the token rows as well (three fewer)
     const PlanView plan = plan_view(base, L);
     int32_t *status = reinterpret_cast<int32_t *>(base + L.status);
+    MOE_STAGE(MOE_STAGE_ROUTER_LOGITS,
+              launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s,
+                                   plan.done_shared, max_shared_segments(T), status));
+    // the grouping kernel also writes the FFN segment plan (one launch fewer); for a small
+    // batch it selects the experts and gathers the token rows as well (three fewer)
     const bool small = route_group_small_applies(*cfg, T);
     if (small) {
         MOE_STAGE(MOE_STAGE_PERMUTE,
@@ -405,10 +427,20 @@ moe_status_t moe_check(void *ws, void *stream)
         return MOE_ERR_INVALID_ARG;
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return MOE_ERR_CUDA;
-    int32_t word = 0;
-    if (cudaMemcpy(&word, ws, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess)
-        return MOE_ERR_CUDA;
-    return word == 0 ? MOE_OK : MOE_ERR_TIMEOUT;
+    return read_and_clear_status(ws);
+}
+
+moe_status_t moe_workspace_region(const moe_config_t *cfg, int32_t T, int32_t index, size_t *offset,
+                                  size_t *bytes)
+{
+    if (check_config(cfg) != MOE_OK || check_tokens(cfg, T) != MOE_OK || !offset || !bytes)
+        return MOE_ERR_INVALID_ARG;
+    const Workspace L = workspace_layout(*cfg, T);
+    if (index < 0 || index >= L.n_regions)
+        return MOE_ERR_INVALID_ARG;
+    *offset = L.region_off[index];
+    *bytes = L.region_bytes[index];
+    return MOE_OK;
 }
 
 moe_status_t moe_selftest_wait_limit(void *ws, int32_t limit_us, void *stream)
@@ -420,7 +452,7 @@ moe_status_t moe_selftest_wait_limit(void *ws, int32_t limit_us, void *stream)
         return st;
     int32_t *status = static_cast<int32_t *>(ws);  // the status region is the first of the workspace
     int launches = 0;
-    MOE_TRY_LAUNCH(launch_wait_limit_selftest(status, status + 1, limit_us,
+    MOE_TRY_LAUNCH(launch_wait_limit_selftest(status, status + 2, limit_us,
                                               static_cast<cudaStream_t>(stream)));
     return MOE_OK;
 }

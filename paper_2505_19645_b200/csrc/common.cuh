@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "device_once.h"
 #include "moe_verify.h"
 
 namespace moe {
@@ -18,6 +19,12 @@ namespace moe {
 // ---------------------------------------------------------------------------------------
 constexpr int SEG_TOKENS = 128;
 constexpr int PLAN_HEADER_INTS = 16;
+
+// Status region (first of the workspace): word [0] is the device status word, raised by a
+// bounded wait that gave up and left alone by everything else until moe_check reads and clears
+// it; word [1] holds STATUS_MAGIC once the region has been initialised (a fresh workspace holds
+// garbage: the first kernel of every call clears word [0] unless the magic is already there).
+constexpr int32_t STATUS_MAGIC = 0x4d6f4553;
 
 struct Segment {
     int32_t expert;     // routed expert id of the group
@@ -56,8 +63,11 @@ __host__ __device__ inline int max_segments(int E, int A) { return E + A / SEG_T
 // ---------------------------------------------------------------------------------------
 // Workspace layout (every region 256-byte aligned).
 // ---------------------------------------------------------------------------------------
+constexpr int WS_MAX_REGIONS = 24;
+constexpr size_t WS_GUARD_BYTES = 256;  // never written: lets a test detect a store that strays
+
 struct Workspace {
-    size_t status;        // int32[64]: [0] device status word
+    size_t status;        // int32[64]: [0] device status word, [1] STATUS_MAGIC once initialised
     size_t logits;        // f32 [T,E]
     size_t topk_idx;      // i32 [T,K]
     size_t topk_w;        // f32 [T,K]
@@ -79,9 +89,31 @@ struct Workspace {
     size_t y;             // bf16 [A, H]      expert outputs, sorted order
     size_t y_shared;      // bf16 [shared_down_parts, T, H]: partial sums per k chunk
     size_t total;
+    // every region in layout order (offset, bytes in use); the bytes between two regions --
+    // the rounding up to 256 and a guard of WS_GUARD_BYTES -- belong to no kernel
+    int n_regions;
+    size_t region_off[WS_MAX_REGIONS], region_bytes[WS_MAX_REGIONS];
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Carves regions off a running offset: 256-byte aligned starts, a guard behind each.
+struct WorkspaceCarver {
+    Workspace &w;
+    size_t off = 0;
+    explicit WorkspaceCarver(Workspace &ws) : w(ws) { w.n_regions = 0; }
+    size_t take(size_t bytes)
+    {
+        const size_t at = off;
+        if (w.n_regions < WS_MAX_REGIONS) {
+            w.region_off[w.n_regions] = at;
+            w.region_bytes[w.n_regions] = bytes;
+            ++w.n_regions;
+        }
+        off = align_up(off + bytes, 256) + WS_GUARD_BYTES;
+        return at;
+    }
+};
 
 // k chunks the shared expert's down projection is split into inside moe_verify_layer (each
 // chunk is a work unit of its own and writes a partial [T,H] plane that the combine step sums)
@@ -97,53 +129,45 @@ inline Workspace workspace_layout(const moe_config_t &c, int T)
 {
     Workspace w{};
     const size_t A = (size_t)T * c.top_k, E = c.n_experts, H = c.hidden;
-    size_t off = 0;
-    auto take = [&](size_t bytes) {
-        size_t at = off;
-        off = align_up(off + bytes, 256);
-        return at;
-    };
-    w.status = take(64 * 4);
-    w.logits = take((size_t)T * E * 4);
-    w.topk_idx = take(A * 4);
-    w.topk_w = take(A * 4);
-    w.shared_scale = take((size_t)T * 4);
-    w.counts = take(E * 4);
-    w.offsets = take((E + 1) * 4);
-    w.active = take(E * 4);
-    w.n_active = take(4);
-    w.perm = take(A * 4);
-    w.inv_perm = take(A * 4);
-    w.plan_header = take(PLAN_HEADER_INTS * 4);
-    w.plan_seg = take(sizeof(Segment) * (size_t)max_segments((int)E, (int)A));
-    w.plan_pairs = take(sizeof(PairEntry) * (size_t)max_segments((int)E, (int)A));
-    w.plan_done = take(4 * ((size_t)max_segments((int)E, (int)A) + max_shared_segments(T)));
+    WorkspaceCarver cut(w);
+    w.status = cut.take(64 * 4);
+    w.logits = cut.take((size_t)T * E * 4);
+    w.topk_idx = cut.take(A * 4);
+    w.topk_w = cut.take(A * 4);
+    w.shared_scale = cut.take((size_t)T * 4);
+    w.counts = cut.take(E * 4);
+    w.offsets = cut.take((E + 1) * 4);
+    w.active = cut.take(E * 4);
+    w.n_active = cut.take(4);
+    w.perm = cut.take(A * 4);
+    w.inv_perm = cut.take(A * 4);
+    w.plan_header = cut.take(PLAN_HEADER_INTS * 4);
+    w.plan_seg = cut.take(sizeof(Segment) * (size_t)max_segments((int)E, (int)A));
+    w.plan_pairs = cut.take(sizeof(PairEntry) * (size_t)max_segments((int)E, (int)A));
+    w.plan_done = cut.take(4 * ((size_t)max_segments((int)E, (int)A) + max_shared_segments(T)));
     w.plan_done_shared_at = (size_t)max_segments((int)E, (int)A);
-    w.x_sorted = take(A * H * 2);
-    w.h = take(A * (size_t)c.inter * 2);
-    w.h_shared = take((size_t)T * c.shared_inter * 2);
+    w.x_sorted = cut.take(A * H * 2);
+    w.h = cut.take(A * (size_t)c.inter * 2);
+    w.h_shared = cut.take((size_t)T * c.shared_inter * 2);
     // y: [A,H], or while the down pass is short of work items partial planes of it
     const size_t A_split = ROUTED_SPLIT_MAX_PARTS * routed_split_max_rows(c, T);
     const size_t y_rows = A > A_split ? A : A_split;
-    w.y = take(y_rows * H * 2);
-    w.y_shared = take((size_t)T * H * 2 * shared_down_parts(c));
-    w.total = off;
+    w.y = cut.take(y_rows * H * 2);
+    w.y_shared = cut.take((size_t)T * H * 2 * shared_down_parts(c));
+    w.total = cut.off;
     return w;
 }
 
 // ---------------------------------------------------------------------------------------
 // Kernel launchers (each enqueues on `stream` and returns the launch error, if any).
 // ---------------------------------------------------------------------------------------
-struct LaunchCounter {
-    int n = 0;
-};
-
 // zero / zero_n: ints this kernel clears before any later kernel of the call may start (the
-// shared expert's progress counters), or null
+// shared expert's progress counters), or null; status: the workspace's status region, which
+// the first kernel of a call initialises if it never was
 cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
                                  const __nv_bfloat16 *x, int T, float *logits,
                                  float *shared_scale, cudaStream_t s, int32_t *zero = nullptr,
-                                 int zero_n = 0);
+                                 int zero_n = 0, int32_t *status = nullptr);
 cudaError_t launch_route_topk(const moe_config_t &c, const float *logits, int T, int32_t *idx,
                               float *wts, cudaStream_t s);
 cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int32_t *counts,
@@ -188,6 +212,9 @@ cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, int ro
 
 int sm_count();
 bool pdl_enabled();  // programmatic dependent launch between the layer's kernels
+// Test hook, read once per process from MOE_FF_RR: 0 / 1 forces the FFN kernels to deal the
+// routed work as ranges / as single items, -1 (unset) leaves the choice to the host heuristic.
+int schedule_override();
 
 // Host-side argument checks and the FFN launch sequence shared by the entry points.
 bool aligned16(const void *p);
@@ -196,6 +223,7 @@ moe_status_t check_tokens(const moe_config_t *c, int64_t T);
 moe_status_t check_device();
 bool weights_ok(const moe_config_t *c, const moe_weights_t *w, bool need_router, bool need_experts);
 PlanView plan_view(char *ws, const Workspace &L);
+moe_status_t read_and_clear_status(void *status_region);
 // plan -> gate/up + SwiGLU -> down; uses the regions status, plan_*, h, h_shared of `L` in `ws`
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,
                      const int32_t *offsets, const int32_t *perm, __nv_bfloat16 *y,
@@ -248,16 +276,6 @@ __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wa
 // Lets the next kernel in the stream start its own prologue.
 __device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// 128-bit streaming load: weights are read exactly once, keep them out of L1.
-__device__ __forceinline__ uint4 ld_stream_v4(const void *p)
-{
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-
 // 128-bit load of data that several warps of the CTA re-read (activations): cache in L1.
 __device__ __forceinline__ uint4 ld_cached_v4(const void *p)
 {
@@ -280,6 +298,15 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
 
 __device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+
+// One thread of the first kernel of a call, after its griddepcontrol.wait.
+__device__ __forceinline__ void status_region_init(int32_t *status)
+{
+    if (status != nullptr && status[1] != STATUS_MAGIC) {
+        status[0] = 0;
+        status[1] = STATUS_MAGIC;
+    }
+}
 
 // g * sigmoid(g) with the fast exponential and division (the result is rounded to bf16)
 __device__ __forceinline__ float silu_f(float g) { return __fdividef(g, 1.0f + __expf(-g)); }

@@ -49,8 +49,9 @@
 // except h, which the down pass takes segment by segment as described above.
 #include <cuda.h>
 #include <math.h>
-#include <stdlib.h>
 #include <string.h>
+
+#include <mutex>
 
 #include "common.cuh"
 
@@ -1102,6 +1103,7 @@ __global__ void wait_limit_selftest_kernel(int32_t *status, int32_t *never_set, 
         abort_flag[0] = 0;
         abort_flag[1] = limit_us;
         status[0] = 0;
+        status[1] = STATUS_MAGIC;
         never_set[0] = 0;
         __threadfence();
         counter_wait(never_set, 1, abort_flag, status);
@@ -1216,6 +1218,65 @@ static bool make_weight_maps(CUtensorMap (&m)[FF_HEIGHTS], const void *base, uin
     return true;
 }
 
+// Encoded tensor maps of recent launches.  A serving loop calls the layer with the same
+// weights, workspace and token count again and again; encoding the twenty maps of a pass costs
+// more host time than the launch itself, so the maps are kept, keyed by everything that enters
+// them (device, pass, base pointers, extents).  A few dozen entries, replaced in turn.
+struct MapKey {
+    int device, gated;
+    const void *ptr[7];
+    uint64_t dim[6];
+};
+struct MapCacheEntry {
+    bool used;
+    MapKey key;
+    FfnMaps maps;
+};
+constexpr int FF_MAP_CACHE = 48;
+static MapCacheEntry g_map_cache[FF_MAP_CACHE];
+static int g_map_cache_next = 0, g_map_cache_last = 0;
+static std::mutex g_map_cache_mutex;
+
+static bool map_cache_lookup(const MapKey &key, FfnMaps &out)
+{
+    std::lock_guard<std::mutex> lock(g_map_cache_mutex);
+    for (int n = 0; n < FF_MAP_CACHE; ++n) {
+        const int i = (g_map_cache_last + n) % FF_MAP_CACHE;  // the last hit first
+        if (g_map_cache[i].used && memcmp(&g_map_cache[i].key, &key, sizeof key) == 0) {
+            out = g_map_cache[i].maps;
+            g_map_cache_last = i;
+            return true;
+        }
+    }
+    return false;
+}
+
+static void map_cache_store(const MapKey &key, const FfnMaps &maps)
+{
+    std::lock_guard<std::mutex> lock(g_map_cache_mutex);
+    MapCacheEntry &e = g_map_cache[g_map_cache_next];
+    e.used = true;
+    e.key = key;
+    e.maps = maps;
+    g_map_cache_last = g_map_cache_next;
+    g_map_cache_next = (g_map_cache_next + 1) % FF_MAP_CACHE;
+}
+
+static MapKey map_key(bool gated, const void *p0, const void *p1, const void *p2, const void *p3,
+                      const void *p4, const void *p5, const void *p6, uint64_t d0, uint64_t d1,
+                      uint64_t d2, uint64_t d3, uint64_t d4, uint64_t d5)
+{
+    MapKey k;
+    memset(&k, 0, sizeof k);  // padding bytes take part in the comparison
+    cudaGetDevice(&k.device);
+    k.gated = gated ? 1 : 0;
+    const void *p[7] = {p0, p1, p2, p3, p4, p5, p6};
+    const uint64_t d[6] = {d0, d1, d2, d3, d4, d5};
+    memcpy(k.ptr, p, sizeof p);
+    memcpy(k.dim, d, sizeof d);
+    return k;
+}
+
 // Expected number of activated experts for T tokens (Eq. N(t): E(1 - (1 - K/E)^T)); the host
 // never sees the routing result, so it sizes rings and shared tiles from the expectation.
 static double expected_active_experts(int E, int k, int T)
@@ -1278,18 +1339,11 @@ static int shared_tile_count(const moe_config_t &c, int T, int rows_routed, int 
 // three 128-row entries otherwise (a pair of segments needs two at once).
 static void ffn_geometry(const moe_config_t &c, int T, FfnArgs &a)
 {
-    const char *ekb = getenv("MOE_FF_KBOXES"), *exr = getenv("MOE_FF_XRING_KB");
-    a.kboxes = ekb ? atoi(ekb) : 2;
+    a.kboxes = 2;
     a.w_slot_bytes = 256 * 128 * a.kboxes;  // a full tile: 256 stacked rows per k box
-    int x_ring_bytes = small_token_ring(c, T) ? 32 * 1024 : 96 * 1024;
-    if (exr)
-        x_ring_bytes = atoi(exr) * 1024;
     // entries never wrap, so two entries that must be resident together (a pair of segments:
     // 32 KB + up to 32 KB) need a ring of three of them wherever the first may sit
-    if (T > FF_SEG && x_ring_bytes < 96 * 1024)
-        x_ring_bytes = 96 * 1024;
-    if (x_ring_bytes < 32 * 1024)
-        x_ring_bytes = 32 * 1024;
+    const int x_ring_bytes = small_token_ring(c, T) ? 32 * 1024 : 96 * 1024;
     a.x_units = x_ring_bytes / FF_X_UNIT;
     const int avail = FF_SMEM_LIMIT - 1024 - 512;  // alignment slack, static shared memory
     int ns = (avail - x_ring_bytes) / a.w_slot_bytes;
@@ -1312,9 +1366,9 @@ static void ffn_geometry(const moe_config_t &c, int T, FfnArgs &a)
 static bool use_round_robin(const moe_config_t &c, int T, int rows_routed, int K_routed, int max_tile,
                             int grid)
 {
-    const char *force = getenv("MOE_FF_RR");
-    if (force)
-        return force[0] == '1';
+    const int force = schedule_override();
+    if (force >= 0)
+        return force == 1;
     const double n_act = expected_active_experts(c.n_experts, c.top_k, T);
     const double rows_per_group = (double)T * c.top_k / n_act;
     const double pairs = n_act * ceil(ceil(rows_per_group / FF_SEG) / 2.0);
@@ -1326,14 +1380,18 @@ static bool use_round_robin(const moe_config_t &c, int T, int rows_routed, int K
 template <bool GATED>
 static cudaError_t launch_ffn(FfnArgs &a, const FfnMaps &maps, cudaStream_t s)
 {
-    static bool configured[2] = {false, false};
-    if (!configured[GATED]) {
+    // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
+    static DeviceOnce configured;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess)
+        return cudaErrorInvalidDevice;
+    if (!configured.done(dev)) {
         cudaError_t e = cudaFuncSetAttribute(ffn_fused_kernel<GATED>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              FF_SMEM_LIMIT - 512);
         if (e != cudaSuccess)
             return e;
-        configured[GATED] = true;
+        configured.mark(dev);
     }
     // the 128-row read of the last token entry may run 16 KB past the token ring: the weight
     // ring behind it is always larger than that
@@ -1361,16 +1419,23 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
                                  : 0;
     ffn_geometry(c, T, a);
     FfnMaps maps;
-    memset(&maps, 0, sizeof maps);
-    bool ok = make_weight_maps(maps.w[0][0], w.w_gate, E * c.inter, H) &&
-              make_weight_maps(maps.w[0][1], w.w_up, E * c.inter, H) &&
-              make_weight_maps(maps.x[0], x_sorted, A, H);
-    if (with_shared)
-        ok = ok && make_weight_maps(maps.w[1][0], w.ws_gate, c.shared_inter, H) &&
-             make_weight_maps(maps.w[1][1], w.ws_up, c.shared_inter, H) &&
-             make_weight_maps(maps.x[1], x, T, H);
-    if (!ok)
-        return cudaErrorInvalidValue;
+    const MapKey key = map_key(true, w.w_gate, w.w_up, x_sorted, with_shared ? w.ws_gate : nullptr,
+                               with_shared ? w.ws_up : nullptr, with_shared ? x : nullptr, nullptr, E,
+                               (uint64_t)c.inter, H, A, with_shared ? (uint64_t)c.shared_inter : 0,
+                               (uint64_t)T);
+    if (!map_cache_lookup(key, maps)) {
+        memset(&maps, 0, sizeof maps);
+        bool ok = make_weight_maps(maps.w[0][0], w.w_gate, E * c.inter, H) &&
+                  make_weight_maps(maps.w[0][1], w.w_up, E * c.inter, H) &&
+                  make_weight_maps(maps.x[0], x_sorted, A, H);
+        if (with_shared)
+            ok = ok && make_weight_maps(maps.w[1][0], w.ws_gate, c.shared_inter, H) &&
+                 make_weight_maps(maps.w[1][1], w.ws_up, c.shared_inter, H) &&
+                 make_weight_maps(maps.x[1], x, T, H);
+        if (!ok)
+            return cudaErrorInvalidValue;
+        map_cache_store(key, maps);
+    }
     a.out[0] = h;
     a.out[1] = h_shared;
     a.out_ld[0] = c.inter;
@@ -1473,14 +1538,21 @@ cudaError_t launch_ffn_down(const moe_config_t &c, const moe_weights_t &w, int T
                                  : 0;
     ffn_geometry(c, T, a);
     FfnMaps maps;
-    memset(&maps, 0, sizeof maps);
-    bool ok = make_weight_maps(maps.w[0][0], w.w_down, E * H, c.inter) &&
-              make_weight_maps(maps.x[0], h, A, c.inter);
-    if (with_shared)
-        ok = ok && make_weight_maps(maps.w[1][0], w.ws_down, H, c.shared_inter) &&
-             make_weight_maps(maps.x[1], h_shared, T, c.shared_inter);
-    if (!ok)
-        return cudaErrorInvalidValue;
+    const MapKey key = map_key(false, w.w_down, h, with_shared ? w.ws_down : nullptr,
+                               with_shared ? h_shared : nullptr, nullptr, nullptr, nullptr, E,
+                               (uint64_t)c.inter, H, A, with_shared ? (uint64_t)c.shared_inter : 0,
+                               (uint64_t)T);
+    if (!map_cache_lookup(key, maps)) {
+        memset(&maps, 0, sizeof maps);
+        bool ok = make_weight_maps(maps.w[0][0], w.w_down, E * H, c.inter) &&
+                  make_weight_maps(maps.x[0], h, A, c.inter);
+        if (with_shared)
+            ok = ok && make_weight_maps(maps.w[1][0], w.ws_down, H, c.shared_inter) &&
+                 make_weight_maps(maps.x[1], h_shared, T, c.shared_inter);
+        if (!ok)
+            return cudaErrorInvalidValue;
+        map_cache_store(key, maps);
+    }
     a.out[0] = y;
     a.out[1] = y_shared;
     a.out_ld[0] = a.out_ld[1] = c.hidden;

@@ -18,7 +18,7 @@ namespace moe {
 static __device__ __align__(256) unsigned char g_static_scratch[MOE_STATIC_SCRATCH_BYTES];
 
 static std::mutex g_scratch_mutex;
-static void *g_scratch_addr[64];  // per device ordinal, resolved on first use
+static void *g_scratch_addr[MAX_DEVICE_ORDINALS];  // per device ordinal, resolved on first use
 
 // Device address of the scratch array on the CURRENT device (resolved once per device).
 static moe_status_t static_scratch_address(char **out)
@@ -26,7 +26,7 @@ static moe_status_t static_scratch_address(char **out)
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess)
         return MOE_ERR_CUDA;
-    if (dev < 0 || dev >= 64)
+    if (dev < 0 || dev >= MAX_DEVICE_ORDINALS)
         return MOE_ERR_UNSUPPORTED;
     std::lock_guard<std::mutex> lock(g_scratch_mutex);
     if (!g_scratch_addr[dev]) {
@@ -44,22 +44,17 @@ static Workspace static_scratch_layout(const moe_config_t &c, int T)
 {
     Workspace w{};
     const size_t A = (size_t)T * c.top_k;
-    size_t off = 0;
-    auto take = [&](size_t bytes) {
-        size_t at = off;
-        off = align_up(off + bytes, 256);
-        return at;
-    };
-    w.status = take(64 * 4);
-    w.plan_header = take(PLAN_HEADER_INTS * 4);
-    w.plan_seg = take(sizeof(Segment) * (size_t)max_segments(c.n_experts, (int)A));
-    w.plan_pairs = take(sizeof(PairEntry) * (size_t)max_segments(c.n_experts, (int)A));
-    w.plan_done = take(4 * ((size_t)max_segments(c.n_experts, (int)A) + max_shared_segments(T)));
+    WorkspaceCarver cut(w);
+    w.status = cut.take(64 * 4);
+    w.plan_header = cut.take(PLAN_HEADER_INTS * 4);
+    w.plan_seg = cut.take(sizeof(Segment) * (size_t)max_segments(c.n_experts, (int)A));
+    w.plan_pairs = cut.take(sizeof(PairEntry) * (size_t)max_segments(c.n_experts, (int)A));
+    w.plan_done = cut.take(4 * ((size_t)max_segments(c.n_experts, (int)A) + max_shared_segments(T)));
     w.plan_done_shared_at = (size_t)max_segments(c.n_experts, (int)A);
-    w.x_sorted = take(A * (size_t)c.hidden * 2);
-    w.h = take(A * (size_t)c.inter * 2);
-    w.h_shared = take((size_t)T * c.shared_inter * 2);
-    w.total = off;
+    w.x_sorted = cut.take(A * (size_t)c.hidden * 2);
+    w.h = cut.take(A * (size_t)c.inter * 2);
+    w.h_shared = cut.take((size_t)T * c.shared_inter * 2);
+    w.total = cut.off;
     return w;
 }
 
@@ -93,12 +88,44 @@ moe_status_t moe_grouped_swiglu_static(const moe_config_t *cfg, const moe_weight
     if ((st = static_scratch_address(&scratch)) != MOE_OK)
         return st;
     int launches = 0;
-    // The plan kernel, first in the sequence, clears the status word and the progress
-    // counters and rewrites the whole plan; the down pass reads a segment of h only once the
-    // gate/up pass has counted it complete.  Nothing else in the array has to start at zero.
+    // The plan kernel, first in the sequence, clears the progress counters and rewrites the
+    // whole plan; the down pass reads a segment of h only once the gate/up pass has counted
+    // it complete.  Nothing else in the array has to start at zero (the status word is
+    // zero when the library is loaded and is cleared by moe_check_static after a report).
     return run_ffn(*cfg, *w, static_cast<const __nv_bfloat16 *>(x), T, offsets, perm,
                    static_cast<__nv_bfloat16 *>(y), static_cast<__nv_bfloat16 *>(shared_y), scratch,
                    L, static_cast<cudaStream_t>(stream), launches);
+}
+
+moe_status_t moe_check_static(void *stream)
+{
+    moe_status_t st = check_device();
+    if (st != MOE_OK)
+        return st;
+    char *scratch = nullptr;
+    if ((st = static_scratch_address(&scratch)) != MOE_OK)
+        return st;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    // the status region is the first of the array (static_scratch_layout)
+    return read_and_clear_status(scratch);
+}
+
+moe_status_t moe_selftest_wait_limit_static(int32_t limit_us, void *stream)
+{
+    if (limit_us < 1 || limit_us > 1000000)
+        return MOE_ERR_INVALID_ARG;
+    moe_status_t st = check_device();
+    if (st != MOE_OK)
+        return st;
+    char *scratch = nullptr;
+    if ((st = static_scratch_address(&scratch)) != MOE_OK)
+        return st;
+    int32_t *status = reinterpret_cast<int32_t *>(scratch);
+    if (launch_wait_limit_selftest(status, status + 2, limit_us, static_cast<cudaStream_t>(stream)) !=
+        cudaSuccess)
+        return MOE_ERR_CUDA;
+    return MOE_OK;
 }
 
 }  // extern "C"

@@ -76,10 +76,8 @@ __device__ void build_plan(const int *cnt_sh, const int *off_sh, int *scan, int 
             plan.done_routed[first + i] = 0;
         }
     }
-    if (tid == 0) {
+    if (tid == 0)
         plan.header[0] = *total;
-        status[0] = 0;  // device status word: cleared at the start of every FFN pass
-    }
     // pairs: segments 2q and 2q+1 of a group
     const int first = nseg > 0 ? scan[tid] : 0;
     const int npair = (nseg + 1) >> 1;
@@ -353,7 +351,6 @@ route_group_small_kernel(const float *__restrict__ logits, const __nv_bfloat16 *
                     plan.header[1] = n_act;  // pairs
                     plan.header[2] = 0;
                     plan.header[3] = 0;
-                    status[0] = 0;
                 }
             }
         } else if (blockIdx.x >= 2) {
@@ -463,6 +460,8 @@ plan_kernel(const int32_t *__restrict__ offsets, int E, int T, int32_t *__restri
     // clear before the gate/up pass, which may start right away, counts on them
     for (int i = threadIdx.x; i < max_shared_segments(T); i += blockDim.x)
         plan.done_shared[i] = 0;
+    if (threadIdx.x == 0)
+        status_region_init(status);
     __threadfence();
     __syncthreads();
     griddep_launch();

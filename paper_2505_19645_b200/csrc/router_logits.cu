@@ -7,7 +7,6 @@
 // m16n8k16 MMAs.  A CTA owns 16 router rows x (8*NCH) tokens; its 16 warps split H and are
 // summed through shared memory, so even T = 1 keeps every load short and parallel.
 #include <cooperative_groups.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -142,15 +141,18 @@ __global__ void __launch_bounds__(RL_WARPS_FOR(NCH) * 32)
 router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ w_router,
                      const float *__restrict__ bias, const __nv_bfloat16 *__restrict__ w_sg,
                      int T, int H, int E, int n_rows, float *__restrict__ logits,
-                     float *__restrict__ shared_scale, int32_t *__restrict__ zero, int zero_n)
+                     float *__restrict__ shared_scale, int32_t *__restrict__ zero, int zero_n,
+                     int32_t *__restrict__ status)
 {
     constexpr int RL_WARPS = RL_WARPS_FOR(NCH);
     __shared__ float part[RL_WARPS][NCH][4][32];
     griddep_wait();    // first kernel of a layer call: everything older is complete from here on
-    if (zero != nullptr && blockIdx.x == 0 && blockIdx.y == 0) {
+    if ((zero != nullptr || status != nullptr) && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
         // counters that a later kernel of this call updates before the plan kernel has run
         for (int i = threadIdx.x; i < zero_n; i += blockDim.x)
             zero[i] = 0;
+        if (threadIdx.x == 0)
+            status_region_init(status);
         __threadfence();
         __syncthreads();
     }
@@ -247,7 +249,8 @@ router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restric
 
 cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
                                  const __nv_bfloat16 *x, int T, float *logits,
-                                 float *shared_scale, cudaStream_t s, int32_t *zero, int zero_n)
+                                 float *shared_scale, cudaStream_t s, int32_t *zero, int zero_n,
+                                 int32_t *status)
 {
     const bool gate_row = shared_scale != nullptr && c.shared_gate && c.shared_inter > 0;
     const int n_rows = c.n_experts + (gate_row ? 1 : 0);
@@ -266,11 +269,7 @@ cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
     // least one step.
     int ks = 1;
     if (nch == 1 && (c.hidden >> 5) / RL_WARPS_FOR(1) >= 8) {
-        static const bool split = [] {
-            const char *e = getenv("MOE_RL_KSPLIT");
-            return !e || atoi(e) != 0;
-        }();
-        ks = split ? 8 : 1;
+        ks = 8;
         while (ks > 1 && ((long long)e_tiles * token_tiles * ks > (long long)sm_count() ||
                           (c.hidden >> 5) / ks < RL_WARPS_FOR(1)))
             ks /= 2;
@@ -278,7 +277,7 @@ cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
     if (ks > 1) {
         grid.z = ks;
         void (*kernel)(const __nv_bfloat16 *, const float *, const float *, const __nv_bfloat16 *, int,
-                       int, int, int, float *, float *, int32_t *, int) = router_logits_kernel<1, 1>;
+                       int, int, int, float *, float *, int32_t *, int, int32_t *) = router_logits_kernel<1, 1>;
         prefer_max_shared_carveout(reinterpret_cast<const void *>(kernel));
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = grid;
@@ -296,13 +295,13 @@ cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
         cfg.numAttrs = 2;
         return cudaLaunchKernelEx(&cfg, kernel, x, w.w_router, w.router_bias,
                                   static_cast<const __nv_bfloat16 *>(w.w_shared_gate), T, c.hidden,
-                                  c.n_experts, n_rows, logits, shared_scale, zero, zero_n);
+                                  c.n_experts, n_rows, logits, shared_scale, zero, zero_n, status);
     }
     const __nv_bfloat16 *w_sg = static_cast<const __nv_bfloat16 *>(w.w_shared_gate);
 #define MOE_RL_LAUNCH(N, R)                                                                 \
     err = launch_pdl(router_logits_kernel<N, R>, grid, dim3(RL_WARPS_FOR(N) * 32), 0, s, x, w.w_router, \
                      w.router_bias, w_sg, T, c.hidden, c.n_experts, n_rows, logits, shared_scale, zero,  \
-                     zero_n)
+                     zero_n, status)
     cudaError_t err = cudaSuccess;
     switch (nch) {
     case 1: MOE_RL_LAUNCH(1, 1); break;

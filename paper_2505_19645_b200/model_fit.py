@@ -158,10 +158,12 @@ def load_sweeps(paths):
     for p in paths:
         line = open(p).read().strip().splitlines()[-1]
         d = json.loads(line)
-        shape = d["config"]["shape"]
-        K, E = shape["top_k"], shape["n_experts"]
-        for pt in d["sweep"]:
-            rows.append((K, pt["gamma"], pt["B"], pt["T"], E, pt["us"]))
+        # every sweep of the line (bench.py --config X --sweeps config carries one)
+        for sw in d["sweeps"].values():
+            shape = sw["shape"]
+            K, E = shape["top_k"], shape["n_experts"]
+            for pt in sw["rows"]:
+                rows.append((K, pt["gamma"], pt["B"], pt["T"], E, pt["us"]))
     rows.sort()
     arr = np.array(rows, dtype=np.float64)
     return {"K": arr[:, 0], "gamma": arr[:, 1], "B": arr[:, 2], "t": arr[:, 3], "E": arr[:, 4],

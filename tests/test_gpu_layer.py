@@ -48,21 +48,44 @@ def test_layer_parity_small_shapes(name, H, E, k, I, Is, score, renorm, sgate, B
     check_layer_against_oracle(shape, w, x, B, gamma)
 
 
-@pytest.mark.parametrize("mode", ["0", "1"])
-@pytest.mark.parametrize("name,H,E,k,I,Is,B,gamma", [
+SCHEDULING_CASES = [
     ("rr-shared", 512, 60, 4, 352, 1408, 13, 4),     # shared expert with a k-split down pass
     ("rr-segments", 256, 4, 2, 384, 256, 100, 3),    # 200 rows per expert: segment pairs, 4 shared segments
     ("rr-ragged", 160, 6, 3, 224, 96, 11, 6),        # tiles shorter than a box, k tails
-])
-def test_layer_parity_in_both_scheduling_modes(monkeypatch, mode, name, H, E, k, I, Is, B, gamma):
-    """The FFN kernels hand out the routed work either as chunks of consecutive tiles or as
-    single (segment pair, tile) items; MOE_FF_RR forces one of the two."""
-    monkeypatch.setenv("MOE_FF_RR", mode)
+]
+
+
+@pytest.mark.parametrize("name,H,E,k,I,Is,B,gamma", SCHEDULING_CASES)
+def test_scheduling_mode_case(name, H, E, k, I, Is, B, gamma):
+    """One case of the scheduling-mode test below (in this process: the host's own choice)."""
     shape = wl.small_shape(name, H, E, k, I, Is, 0, 0, 1)
     w = wl.make_weights(shape, 300 + E, "cuda")
     T = B * (gamma + 1)
     x = wl.make_tokens(shape, T, 400 + T, "cuda")
     check_layer_against_oracle(shape, w, x, B, gamma)
+
+
+def _run_child(env_extra, k_expr):
+    import os
+    import subprocess
+    import sys
+
+    env = dict(os.environ, **env_extra)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run(
+        [sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_layer.py"), "-q", "-x",
+         "-m", "gpu", "-k", k_expr],
+        env=env, cwd=root, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+    assert "passed" in r.stdout
+
+
+@pytest.mark.parametrize("mode", ["0", "1"])
+def test_layer_parity_in_both_scheduling_modes(mode):
+    """The FFN kernels hand out the routed work either as chunks of consecutive tiles or as
+    single (segment pair, tile) items; MOE_FF_RR (a test hook the library reads once per
+    process) forces one of the two, so the cases run in a child process per mode."""
+    _run_child({"MOE_FF_RR": mode}, "scheduling_mode_case")
 
 
 def test_layer_depends_on_token_count_only_and_is_deterministic():
@@ -114,33 +137,26 @@ def test_layer_parity_with_plain_stream_ordering():
     """MOE_NO_PDL=1 (read once per process) launches every kernel with plain stream ordering:
     the kernels then run one after the other and every progress counter is complete when its
     reader starts.  Runs a few of the cases above in a child process."""
-    import os
-    import subprocess
-    import sys
-
-    env = dict(os.environ, MOE_NO_PDL="1")
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    r = subprocess.run(
-        [sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_layer.py"), "-q", "-x",
-         "-m", "gpu", "-k", "small_shapes and (qwen-like or mixtral-like or ksplit-routed)"],
-        env=env, cwd=root, capture_output=True, text=True, timeout=600)
-    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
-    assert "passed" in r.stdout
+    _run_child({"MOE_NO_PDL": "1"},
+               "small_shapes and (qwen-like or mixtral-like or ksplit-routed)")
 
 
 def test_wait_limit_expiry_is_reported_and_the_context_stays_usable():
     """Every wait inside the kernels has a limit.  The self-test runs the down pass's wait for
     a progress counter on a word nothing sets: it gives up after its limit, the kernel raises
     the workspace's status word and returns, moe_check reports MOE_ERR_TIMEOUT, nothing
-    faults, and the same workspace serves a correct layer call right after."""
+    faults, and the same workspace serves a correct layer call right after.  The word is
+    sticky: a layer call enqueued behind the failed wait does not erase the report, and the
+    report is made exactly once."""
     import time
     from paper_2505_19645_b200 import api
 
     shape = wl.small_shape("limit", 512, 60, 4, 352, 1408, 0, 0, 1)
     w = wl.make_weights(shape, 160, "cuda")
     x = wl.make_tokens(shape, 65, 265, "cuda")
-    cfg = api.make_config(shape)
+    cfg, cw = api.make_config(shape), api.make_weights(w)
     ws = api.alloc_workspace(cfg, 65)
+    api.moe_check(ws)   # a workspace no call has touched yet reports nothing
     run_gpu_layer(shape, w, x, 13, 4, ws=ws)
     t0 = time.perf_counter()
     api.moe_selftest_wait_limit(ws, 20000)  # 20 ms
@@ -149,44 +165,102 @@ def test_wait_limit_expiry_is_reported_and_the_context_stays_usable():
     waited = time.perf_counter() - t0
     assert err.value.status == 5  # MOE_ERR_TIMEOUT
     assert 0.015 < waited < 1.0
-    out, _ = run_gpu_layer(shape, w, x, 13, 4, ws=ws)   # clears the status word, runs normally
+    api.moe_check(ws)   # reported once
+    # a failure in an earlier call of a queue is still seen after later calls
+    out = torch.empty_like(x)
+    api.moe_selftest_wait_limit(ws, 2000)
+    api.moe_verify_layer(cfg, cw, x, 13, 4, out, ws)
+    api.moe_verify_layer(cfg, cw, x, 13, 4, out, ws)
+    with pytest.raises(api.MoeError) as err:
+        api.moe_check(ws)
+    assert err.value.status == 5
+    out, _ = run_gpu_layer(shape, w, x, 13, 4, ws=ws)   # runs normally, nothing to report
     ref, _ = run_gpu_layer(shape, w, x, 13, 4)
     assert torch.equal(out, ref)
     check_layer_against_oracle(shape, w, x, 13, 4)
 
 
 # ---- full-size shapes in the launch configuration the benchmark times -------------------
-# The oracle evaluates a seeded sample of token rows (the layer is token-wise, so a row
-# check is exact); routing and grouping are checked on every token.
+# Routing and grouping are checked on every token; the outputs on 16 token rows that the
+# oracle evaluates one by one (the layer is token-wise, so a row check is exact).  The rows
+# are not drawn at random: they are picked from the grouping so that the first and last row of
+# the largest group, a ragged tail segment, both sides of a segment boundary and the ends of
+# the shared expert's last segment pair are always among them (parity_utils.stratified_rows).
 
-def _full_size(name, B, gamma, n_rows, zipf=None):
+_FULL = {}   # weights of one config at a time, on the device and on the host
+N_ROWS = 16
+
+
+def _full_weights(name, zipf):
+    if _FULL.get("name") != name:
+        _FULL.clear()
+        torch.cuda.empty_cache()
+        shape = wl.CONFIGS[name]
+        need = 2.2 * 6 * shape.hidden * shape.inter * shape.n_experts   # bytes, with head room
+        free, _ = torch.cuda.mem_get_info()
+        import psutil
+        if free < need or psutil.virtual_memory().available < need:
+            pytest.skip("needs %.0f GB of device and of host memory" % (need / 1e9))
+        w = wl.make_weights(shape, wl.config_seed(name), "cuda")
+        _FULL.update(name=name, dev=w, host=to_host(w))
+    w_dev, w_host = dict(_FULL["dev"]), dict(_FULL["host"])
+    if zipf is not None:   # the skew variant differs in the router bias only
+        shape = wl.CONFIGS[name]
+        b = wl.zipf_router_bias(shape.n_experts, shape.hidden, zipf, wl.config_seed(name), "cpu")
+        w_host["router_bias"] = b
+        w_dev["router_bias"] = b.cuda()
+    return w_dev, w_host
+
+
+def _full_size(name, B, gamma, zipf=None):
     shape = wl.CONFIGS[name]
-    w = wl.make_weights(shape, wl.config_seed(name), "cuda", zipf_s=zipf)
+    w_dev, w_host = _full_weights(name, zipf)
     T = B * (gamma + 1)
     x = wl.make_tokens(shape, T, wl.point_seed(name, B, gamma), "cuda")
-    rng = np.random.default_rng(T)
-    rows = sorted(rng.choice(T, size=min(n_rows, T), replace=False).tolist())
-    return check_layer_against_oracle(shape, w, x, B, gamma, rows=rows)
+    fr, dbg = check_layer_against_oracle(shape, w_dev, x, B, gamma, rows=N_ROWS, w_host=w_host)
+    return fr, dbg
 
 
-@pytest.mark.parametrize("B,gamma", [(1, 0), (4, 1), (32, 3), (128, 4), (1024, 3)])
+def test_zipf_bias_is_the_only_difference_of_the_skew_variant():
+    shape = wl.small_shape("zb", 64, 16, 2, 64)
+    a = wl.make_weights(shape, 3, "cuda")
+    b = wl.make_weights(shape, 3, "cuda", zipf_s=1.1)
+    for key in a:
+        if key != "router_bias":
+            assert (a[key] is None and b[key] is None) or torch.equal(a[key], b[key])
+    assert torch.equal(b["router_bias"].cpu(), wl.zipf_router_bias(16, 64, 1.1, 3, "cpu"))
+
+
+@pytest.mark.parametrize("B,gamma", [(1, 0), (4, 0), (4, 1), (32, 3), (128, 4), (1024, 3)])
 def test_full_size_qwen15_shape(B, gamma):
-    _full_size("qwen1.5-moe-a2.7b", B, gamma, 6)
+    _full_size("qwen1.5-moe-a2.7b", B, gamma)
 
 
-@pytest.mark.parametrize("B,gamma,zipf", [(8, 2, None), (64, 4, 1.2), (256, 4, None)])
+@pytest.mark.parametrize("B,gamma,zipf", [(1, 0, None), (8, 2, None), (64, 4, 1.2), (256, 4, None),
+                                          (256, 4, 1.2), (512, 3, None), (1024, 3, None)])
 def test_full_size_qwen2_57b_shape(B, gamma, zipf):
-    _full_size("qwen2-57b-a14b", B, gamma, 3, zipf)
+    """Up to the top of the config's grid (T = 1280, also with Zipf(1.2) popularity) and the two
+    extra token counts 2048 and 4096."""
+    _full_size("qwen2-57b-a14b", B, gamma, zipf)
 
 
-@pytest.mark.parametrize("B,gamma", [(16, 2), (256, 4)])
+@pytest.mark.parametrize("B,gamma", [(1, 0), (16, 2), (256, 4)])
 def test_full_size_mixtral_shape(B, gamma):
-    _full_size("mixtral-8x7b", B, gamma, 3)
+    _full_size("mixtral-8x7b", B, gamma)
 
 
-def test_full_size_deepseek_v3_shape():
-    free, _ = torch.cuda.mem_get_info()
-    import psutil
-    if free < 40e9 or psutil.virtual_memory().available < 40e9:
-        pytest.skip("needs 40 GB of device and host memory")
-    _full_size("deepseek-v3", 16, 3, 3)
+@pytest.mark.parametrize("B,gamma,zipf", [(1, 0, None), (16, 3, None), (128, 3, None), (64, 3, 1.0),
+                                          (512, 5, None), (512, 5, 1.0), (512, 3, None),
+                                          (1024, 3, None)])
+def test_full_size_deepseek_v3_shape(B, gamma, zipf):
+    """The largest shape (22.6 GB of expert weights): bottom, middle and top (T = 3072) of its
+    grid, the Zipf(1.0) variant in the middle and at the top, and T = 2048 / 4096."""
+    fr, dbg = _full_size("deepseek-v3", B, gamma, zipf)
+    if zipf is not None and B * (gamma + 1) >= 256:
+        # skew shows: the most popular expert holds several times the mean share
+        assert dbg["counts"].max() > 3 * dbg["counts"].mean()
+
+
+def test_full_size_weights_are_released():
+    _FULL.clear()
+    torch.cuda.empty_cache()

@@ -100,3 +100,53 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(api, "LIB_PATH", os.path.join(ROOT, "no_such_dir", "libmoe_verify.so"))
     with pytest.raises(ImportError):
         api.load_library()
+
+
+def test_workspace_regions_are_disjoint_aligned_and_guarded():
+    """Every region starts 256-byte aligned, lies inside moe_workspace_bytes and is followed
+    by at least 256 bytes that belong to no region (the canary gaps of the GPU tests)."""
+    from paper_2505_19645_b200 import api
+
+    for name, T in (("tiny", 16), ("qwen1.5-moe-a2.7b", 1), ("qwen2-57b-a14b", 1280),
+                    ("deepseek-v3", 3072)):
+        cfg = api.make_config(wl.CONFIGS[name])
+        total = api.moe_workspace_bytes(cfg, T)
+        regions = api.workspace_regions(cfg, T)
+        assert len(regions) == 20
+        end = 0
+        for i, (off, n) in enumerate(regions):
+            assert off % 256 == 0
+            assert off >= end + (256 if i else 0), (name, i)
+            end = off + n
+        assert end + 256 <= total
+        assert regions[0] == (0, 256)   # the status region leads the workspace
+
+
+def test_per_device_set_up_state_is_kept_per_ordinal(tmp_path):
+    """State the CUDA runtime keeps per device (the FFN kernels' shared-memory opt-in, the
+    address of the built-in scratch array) is tracked per device ordinal by DeviceOnce: marking
+    one ordinal must not mark another.  Compiled from the library's own header."""
+    import subprocess
+
+    src = tmp_path / "once.cpp"
+    src.write_text('''
+#include "device_once.h"
+int main() {
+    moe::DeviceOnce once;
+    if (once.done(0) || once.done(1)) return 1;
+    once.mark(0);
+    if (!once.done(0)) return 2;
+    if (once.done(1)) return 3;          // a second GPU still needs its own set-up
+    once.mark(1);
+    if (!once.done(1) || !once.done(0)) return 4;
+    once.mark(-1); once.mark(1000);       // out of the table: ignored, never "done"
+    if (once.done(-1) || once.done(1000)) return 5;
+    moe::DeviceOnce other;
+    if (other.done(0)) return 6;          // one object per piece of state
+    return 0;
+}
+''')
+    exe = tmp_path / "once"
+    subprocess.run(["g++", "-std=c++17", "-I", os.path.join(ROOT, "paper_2505_19645_b200", "csrc"),
+                    str(src), "-o", str(exe)], check=True)
+    assert subprocess.run([str(exe)]).returncode == 0
