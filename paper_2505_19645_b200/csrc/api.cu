@@ -62,6 +62,15 @@ int schedule_override()
     return v;
 }
 
+int geometry_override()
+{
+    static const int v = [] {
+        const char *e = getenv("MOE_FF_WIDE");
+        return !e ? -1 : (e[0] == '1' ? 1 : (e[0] == '0' ? 0 : -1));
+    }();
+    return v;
+}
+
 static thread_local int g_last_launches = 0;
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -172,9 +181,9 @@ moe_status_t read_and_clear_status(void *status_region)
     return MOE_ERR_TIMEOUT;
 }
 
-PlanView plan_view(char *ws, const Workspace &L)
+PlanView plan_view(char *ws, const Workspace &L, int seg_rows)
 {
-    return PlanView{reinterpret_cast<int32_t *>(ws + L.plan_header),
+    return PlanView{seg_rows, reinterpret_cast<int32_t *>(ws + L.plan_header),
                     reinterpret_cast<Segment *>(ws + L.plan_seg),
                     reinterpret_cast<PairEntry *>(ws + L.plan_pairs),
                     reinterpret_cast<int32_t *>(ws + L.plan_done),
@@ -188,7 +197,7 @@ moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_b
                      bool gathered)
 {
     const bool with_shared = shared_y != nullptr && c.shared_inter > 0;
-    const PlanView plan = plan_view(ws, L);
+    const PlanView plan = plan_view(ws, L, ffn_segment_rows(c, T));
     int32_t *status = reinterpret_cast<int32_t *>(ws + L.status);
     __nv_bfloat16 *h = reinterpret_cast<__nv_bfloat16 *>(ws + L.h);
     __nv_bfloat16 *hs = reinterpret_cast<__nv_bfloat16 *>(ws + L.h_shared);
@@ -370,7 +379,7 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
         Arm() { g_probe_armed = true; }
         ~Arm() { g_probe_armed = false; }
     } arm;
-    const PlanView plan = plan_view(base, L);
+    const PlanView plan = plan_view(base, L, ffn_segment_rows(*cfg, T));
     int32_t *status = reinterpret_cast<int32_t *>(base + L.status);
     MOE_STAGE(MOE_STAGE_ROUTER_LOGITS,
               launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s,

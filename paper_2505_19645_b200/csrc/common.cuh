@@ -11,7 +11,8 @@ namespace moe {
 
 // ---------------------------------------------------------------------------------------
 // Segment plan.  The token rows of an activated expert (a "group") are cut into segments of
-// at most SEG_TOKENS consecutive sorted rows, the M extent of one tensor-core instruction.
+// at most SEG_TOKENS (or, for calls whose groups run to hundreds of rows, 2 * SEG_TOKENS)
+// consecutive sorted rows, the N extent of one tensor-core instruction.
 // The plan lists one entry per segment; every entry carries its whole group, so that any
 // segment index leads to the group, its first segment and its number of segments.  The plan
 // is derived from the grouping offsets on the device: the host never needs the
@@ -33,21 +34,21 @@ struct Segment {
     int32_t first_seg;  // plan index of the group's first segment
 };
 
-// plan header (ints): [0] number of segments over all activated experts,
-//                     [1] number of segment pairs (segments 2q and 2q+1 of a group form a pair),
+// plan header (ints): [0] number of segments over all activated experts, [1] the same,
 //                     [2], [3] routed work claimed so far by the gate/up and the down pass
-// A pair of segments (2q, 2q+1) of one group, with the group itself: everything a CTA needs to
-// start on a (pair, tile) item in one 32-byte load.
+// A segment with its group: everything a CTA needs to start on a (segment, tile) item in one
+// 32-byte load.
 struct __align__(16) PairEntry {
     int32_t expert, row0, n, first_seg;  // the group (as in Segment)
-    int32_t seg;                         // plan index of the pair's first segment
+    int32_t seg;                         // plan index of the segment
     int32_t pad[3];
 };
 
 struct PlanView {
+    int seg_rows;         // token rows per segment: SEG_TOKENS or twice that (set by the host)
     int32_t *header;      // written by the plan; [2], [3] advanced by the FFN kernels
     Segment *seg;         // capacity max_segments()
-    PairEntry *pairs;     // one entry per pair of segments, capacity max_segments()
+    PairEntry *pairs;     // one entry per segment (with its group), capacity max_segments()
     // Progress of the gate/up pass, read by the down pass: 16-row units of h written so far
     // (counted once per epilogue warp) for every routed segment [max_segments()] and for
     // every 128-row segment of the shared expert [max_shared_segments()].
@@ -215,6 +216,11 @@ bool pdl_enabled();  // programmatic dependent launch between the layer's kernel
 // Test hook, read once per process from MOE_FF_RR: 0 / 1 forces the FFN kernels to deal the
 // routed work as ranges / as single items, -1 (unset) leaves the choice to the host heuristic.
 int schedule_override();
+// The same for the ring geometry, from MOE_FF_WIDE: 0 / 1 forces segments of 128 / 256 rows.
+int geometry_override();
+// Token rows per segment of the routed groups for a call with T tokens: 128 or 256 (the plan and
+// the FFN kernels of one call must agree on it).
+int ffn_segment_rows(const moe_config_t &c, int T);
 
 // Host-side argument checks and the FFN launch sequence shared by the entry points.
 bool aligned16(const void *p);
@@ -222,7 +228,7 @@ moe_status_t check_config(const moe_config_t *c);
 moe_status_t check_tokens(const moe_config_t *c, int64_t T);
 moe_status_t check_device();
 bool weights_ok(const moe_config_t *c, const moe_weights_t *w, bool need_router, bool need_experts);
-PlanView plan_view(char *ws, const Workspace &L);
+PlanView plan_view(char *ws, const Workspace &L, int seg_rows);
 moe_status_t read_and_clear_status(void *status_region);
 // plan -> gate/up + SwiGLU -> down; uses the regions status, plan_*, h, h_shared of `L` in `ws`
 moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x, int T,

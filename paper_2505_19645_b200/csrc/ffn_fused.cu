@@ -2,43 +2,50 @@
 // experts' weights are streamed from HBM exactly once by TMA through a ring of shared-memory
 // slots and contracted on the tensor cores (tcgen05.mma, fp32 accumulators in TMEM).
 //
-// Orientation.  A tcgen05.mma of shape M x N x 16 occupies the tensor pipe for about M cycles
-// whatever N is (measured: 146 cycles for M = 128 and any N from 16 to 256).  The weight tile
-// is therefore the N operand (up to 256 rows per instruction: a gate tile and the matching up
-// tile stacked, or 256 rows of W_down) and the group's token rows are the M operand (128 TMEM
-// lanes, of which only the first n carry tokens; the remaining lanes compute on stale shared
-// memory and are never read).  One instruction then retires 8 KB of weights, far more than
-// HBM delivers per SM in that time, so the kernel stays bandwidth-bound from one token per
-// expert up to the roofline ridge (Sec. 3.3: the layer's time is the time to load the
-// activated experts), and at 128 tokens per segment the same instruction runs at full rate.
+// Orientation.  Measured on this part, one tcgen05.mma kind::f16 of shape M x N x 16 occupies
+// the tensor pipe for max(48.5, N / 2) cycles, whatever M in {64, 128} is and whether or not
+// consecutive instructions share an accumulator.  The weight rows are therefore the M operand
+// (blocks of 128 rows: a gate block and the matching up block, or two blocks of W_down) and the
+// group's token rows are the N operand (a segment of up to 128 or 256 rows, rounded up to 16):
+// the instruction time follows the number of tokens, so a group of 160 rows costs 160/256 of a
+// full tile instead of two full instructions, and a handful of tokens cost the 48.5-cycle floor
+// -- 8 KB of weights per 97 cycles, far more than HBM delivers per SM in that time.  The kernel
+// stays bandwidth-bound from one token per expert up to the roofline ridge (Sec. 3.3: the
+// layer's time is the time to load the activated experts), and full 256-token segments run the
+// instruction at its full rate.  In TMEM a lane is a weight row (an output feature) and a
+// column a token: an epilogue thread owns one feature and walks the tokens.
 //
 // Work partition.  Output features are independent, so the weight rows of all routed
-// groups are laid end to end (one position = 16 rows of one group for one of its 128-row
-// segments) and the CTAs of the persistent grid claim chunks of positions at run time from a
-// grid-wide counter (chunk ends on tile boundaries, sizes shrinking as the work runs out), or,
-// where chunks would be too short or too many, single (segment pair, tile, k chunk) items: a
-// CTA that starts late or runs slowly takes less, there is no tile-count quantisation and no
-// tail wave.  The shared expert's rows are cut into (tile, k chunk, segment pair) units that
-// are dealt round-robin to the CTAs; they depend on nothing the layer computes, so they run
-// before the routing result exists.  Tiles have at most 128 (gate/up) or 256 (down) rows.  A
-// group with more than 128 token rows has several segments; two segments share one pass over
-// a tile (the weight slot is multiplied with both, one accumulator buffer each), and the
-// units of one shared tile run at the same time on neighbouring CTAs and meet in L2.
+// groups are laid end to end (one position = 16 rows of one group for one of its segments)
+// and the CTAs of the persistent grid claim chunks of positions at run time from a grid-wide
+// counter (chunk ends on tile boundaries, sizes shrinking as the work runs out), or, where
+// chunks would be too short or too many, single (segment, tile, k chunk) items: a CTA that
+// starts late or runs slowly takes less, there is no tile-count quantisation and no tail wave.
+// The shared expert's rows are cut into (tile, k chunk, segment) units that are dealt
+// round-robin to the CTAs; they depend on nothing the layer computes, so they run before the
+// routing result exists.  Tiles have at most 128 features (gate/up: two blocks, gate and up)
+// or 256 (down: two blocks).  The units of one shared tile run at the same time on
+// neighbouring CTAs and meet in L2.
 //
 // Between the passes.  The gate/up pass counts, per segment, the 16-column units of h its
 // epilogue warps have stored (a releasing reduction); the down pass starts while the gate/up
 // pass is still running and fetches a segment's rows of h once the segment's count is
 // complete (acquire load, then a proxy fence before the TMA loads).
 //
-// A weight slot of the shared-memory ring holds two 64-element k boxes of one tile (64 KB
-// for a full tile), so that one producer/consumer hand-shake moves enough bytes to keep HBM
-// busy and every weight row is requested in 256 contiguous bytes; the token operand lives in
-// a second ring whose entries are sized by the segment's row count and never wrap.
+// Two ring geometries, chosen by the host per call.  Streaming (segments of up to 128 rows): a
+// weight slot holds two 64-element k boxes of one tile (64 KB for a full tile), so that one
+// producer/consumer hand-shake moves enough bytes to keep HBM busy and every weight row is
+// requested in 256 contiguous bytes; two sets of accumulators, so the epilogue of one tile
+// runs under the instructions of the next.  Contraction (segments of up to 256 rows, for
+// groups in the hundreds of rows): one k box per slot (32 KB) and per token entry (up to
+// 32 KB), four weight slots and three token entries, one set of accumulators of 2 x 256
+// columns.  The token operand lives in a second ring whose entries are sized by the
+// segment's row count and never wrap.
 //
 // CTA = 7 warps.  warp 0: weight producer (one lane issues TMA), warp 1: MMA issuer (one
 // lane) and owner of the TMEM allocation, warp 2: token-operand producer, warps 3..6:
 // epilogue (tcgen05.ld of one TMEM lane quarter each, SwiGLU, bf16 store).  Rings and the
-// two accumulator buffers are handed over through mbarriers.  Every wait is bounded: when one
+// accumulator sets are handed over through mbarriers.  Every wait is bounded: when one
 // gives up it raises the CTA's abort flag and the device status word, all roles leave their
 // loops, TMEM is freed and the kernel returns.
 //
@@ -60,7 +67,8 @@ namespace moe {
 constexpr int FF_THREADS = 224;
 constexpr int FF_MAX_W_SLOTS = 8;
 constexpr int FF_X_ENTRIES = 8;                               // token-ring entries in flight
-constexpr int FF_SEG = SEG_TOKENS;                            // token rows per segment (MMA M)
+constexpr int FF_SEG = SEG_TOKENS;        // token rows per segment in the streaming geometry
+constexpr int FF_SEG_WIDE = 2 * SEG_TOKENS;  // ... in the contraction geometry (the MMA's N limit)
 constexpr uint64_t FF_WAIT_NS = 1000ull * 1000ull * 1000ull;  // 1 s per wait
 constexpr int FF_TMEM_COLS = 512;
 constexpr int FF_SMEM_LIMIT = 227 * 1024;
@@ -72,9 +80,9 @@ struct FfnArgs {
     int K[2];      // reduction length per group kind
     __nv_bfloat16 *out[2];
     int out_ld[2];
-    const int32_t *plan_header;  // [0] = number of segments, [1] = number of segment pairs
+    const int32_t *plan_header;  // [0] = [1] = number of segments
     const Segment *seg;
-    const PairEntry *pairs;      // the segment pairs with their groups
+    const PairEntry *pairs;      // one entry per segment, with its group
     int32_t *claim_counter;      // grid-wide: next unclaimed routed position / item of this pass
     int32_t *done[2];            // per segment of each group kind: 16-column units of h finished
                                  // by the gate/up pass, summed over its four epilogue warps
@@ -90,7 +98,7 @@ struct FfnArgs {
     int routed_ksplit;   // the same for the routed groups (round-robin mode of the down pass only)
     int routed_kchunk;
     long long routed_part_stride;
-    int shared_tiles;  // tiles of the shared expert's rows; (tile, segment pair) units are dealt
+    int shared_tiles;  // tiles of the shared expert's rows; (tile, k chunk, segment) units are dealt
                        // round-robin to the CTAs; the first (units % tiles) tiles have one
                        // 16-row unit more
     int max_tile;      // weight rows per tile: 128 (gate + up stacked) or 256 (down)
@@ -99,10 +107,11 @@ struct FfnArgs {
     int n_w_slots;
     int x_units;       // token ring size in FF_X_UNIT units
     int wait_us;       // limit of every wait inside the kernel, microseconds
-    int shared_seg;    // token rows per segment of the shared expert: FF_SEG, or half of it
-                       // for 64 < T <= 128, where two 64-row segments are run as single items so
-                       // that no token entry exceeds 16 KB and the ring can be small
-    int shared_paired; // two segments of the shared expert share one pass over a tile
+    int seg_rows;      // token rows per segment of the routed groups (as in the plan): 128 or 256
+    int shared_seg;    // token rows per segment of the shared expert: seg_rows, or 64 for
+                       // 64 < T <= 128 with the small token ring (no entry beyond 16 KB)
+    int acc_sets;      // accumulator sets in TMEM: 2 (segments up to 128 rows: a set is 2 x 128
+                       // columns) or 1 (up to 256 rows: 2 x 256 columns)
 };
 
 // Tensor maps of one pass: weights [kind][matrix][box height], token operand [kind][box height].
@@ -267,6 +276,40 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
         : "memory");
 }
 
+// The same, always accumulating (no predicate to derive from a register).
+__device__ __forceinline__ void umma_bf16_acc(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                              uint32_t idesc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.eq.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        :
+        : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
+        : "memory");
+}
+
+// The instructions of one 64-element k box: four k steps of 16, each against NBLK weight blocks
+// that share the step's token slice.  The issuing thread is the only one that feeds the tensor
+// pipe, so this is straight-line code: descriptors advance by adding to their address field
+// (16-byte units; a 32-byte k step is +2), and only the very first instruction of an item
+// carries a run-time accumulate flag.
+template <int NBLK>
+__device__ __forceinline__ void issue_k_box(uint32_t d0, uint32_t acc_block, uint64_t w_desc,
+                                            uint32_t w_blk16, uint64_t x_desc, uint32_t idesc,
+                                            uint32_t accum_first)
+{
+#pragma unroll
+    for (int m = 0; m < NBLK; ++m)
+        umma_bf16(d0 + m * acc_block, w_desc + (uint64_t)(m * w_blk16), x_desc, idesc, accum_first);
+#pragma unroll
+    for (int q = 1; q < 4; ++q)
+#pragma unroll
+        for (int m = 0; m < NBLK; ++m)
+            umma_bf16_acc(d0 + m * acc_block, w_desc + (uint64_t)(m * w_blk16 + 2 * q),
+                          x_desc + (uint64_t)(2 * q), idesc);
+}
+
 // Arrives on the mbarrier when every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
@@ -315,18 +358,15 @@ __device__ __forceinline__ uint32_t umma_idesc_bf16(int n)
 // ---- kernel ----------------------------------------------------------------------------
 
 // One work item: one segment of token rows of a group against one tile of its weight rows.
-// Two segments of the same group run as a pair on one pass over the tile: the weight slot is
-// loaded once and multiplied with both segments' rows into the two accumulator buffers.
 struct Item {
     int grp;     // 0 routed, 1 shared
     int expert;  // routed expert id (0 for the shared expert)
     int f0;      // first output feature (weight row inside the expert), multiple of 16
-    int h;       // weight rows of the tile, multiple of 16
+    int h;       // output features of the tile, multiple of 16
     int row0;    // first token row (sorted row for routed groups, token for the shared expert)
-    int n;       // token rows, 1..FF_SEG
-    int role;    // 0 single, 1 first of a pair, 2 second of a pair (shares the first's tile)
+    int n;       // token rows, 1..seg_rows
     int seg;     // index of the segment's progress counter (plan index; shared: segment number)
-    int w_once;  // the tile's weights are read by this item (or pair) only
+    int w_once;  // the tile's weights are read by this item only
     int k0, k1;  // reduction range [k0, k1)
     long long out_off;  // element offset of this item's output plane (k chunk) in out[grp]
 };
@@ -354,9 +394,9 @@ struct ClaimRing {
 // Routed work, range mode: positions (16 rows of one group for one of its segments, groups
 // laid end to end); a chunk is a run of positions whose ends are moved to tile boundaries, its
 // length shrinks as the work runs out (a third of the remaining per-CTA share, at least one
-// tile).  Round-robin mode: a chunk is one (segment pair, tile) item; consecutive items are
-// the tiles of one pair, which then run on many CTAs at once and share the pair's token rows
-// in L2.
+// tile).  Round-robin mode: a chunk is one (segment, tile, k chunk) item; consecutive items are
+// the tiles of one segment, which then run on many CTAs at once and share the segment's token
+// rows in L2.
 struct ItemWalk {
     const FfnArgs &a;
     const ClaimRing &ring;
@@ -365,8 +405,8 @@ struct ItemWalk {
     const bool warp_wide;  // the role is run by all 32 lanes in lock step (epilogue warps)
     const int max_units;
     int n_claims;
-    // shared expert: units (tile, k chunk, segment pair) sj, sj + grid, ...
-    int sj, Us, s_base, s_rem, nseg_s, pairs_s, s_units;
+    // shared expert: units (tile, k chunk, segment) sj, sj + grid, ...
+    int sj, Us, s_base, s_rem, nseg_s, s_units;
     // routed groups: current chunk from (fs, u) to (fs_hi, u_hi); fs = plan index of a
     // group's first segment
     int R0, nseg_total, fs, u, fs_hi, u_hi;
@@ -378,7 +418,7 @@ struct ItemWalk {
     Segment sg;
     int g_nseg, g_u_end;
     bool have_tile;
-    int t_grp, t_expert, t_u0, t_h, t_row0, t_n, t_s, t_s_end, t_seg0, t_s0, t_seg_rows;
+    int t_grp, t_expert, t_u0, t_h, t_row0, t_n, t_s, t_s_end, t_seg0, t_seg_rows;
     bool t_once;  // the tile's weights are read by this pass over it only
     int t_k0, t_k1;
     long long t_out_off;
@@ -396,8 +436,7 @@ struct ItemWalk {
         s_rem = a.shared_tiles ? Us % a.shared_tiles : 0;
         sj = blockIdx.x;
         nseg_s = (a.T + a.shared_seg - 1) / a.shared_seg;
-        pairs_s = a.shared_paired ? (nseg_s + 1) >> 1 : nseg_s;
-        s_units = a.shared_tiles * a.shared_ksplit * pairs_s;
+        s_units = a.shared_tiles * a.shared_ksplit * nseg_s;
         R0 = a.rows[0] >> 4;
         nseg_total = fs = u = fs_hi = u_hi = 0;
         ntiles = (R0 + max_units - 1) / max_units;
@@ -414,7 +453,7 @@ struct ItemWalk {
             return;
         }
         const Segment s = a.seg[(int)(p / R0)];
-        const int ns = (s.n + FF_SEG - 1) / FF_SEG;
+        const int ns = (s.n + a.seg_rows - 1) / a.seg_rows;
         fs_out = s.first_seg;
         u_out = (int)((p - (long long)s.first_seg * R0) / ns) / max_units * max_units;
     }
@@ -535,8 +574,6 @@ struct ItemWalk {
                     it.h = t_h << 4;
                     it.row0 = t_row0 + t_s * t_seg_rows;
                     it.n = min(t_seg_rows, t_n - t_s * t_seg_rows);
-                    // the segments of a tile pair up from its first one on
-                    it.role = ((t_s - t_s0) & 1) ? 2 : (t_s + 1 < t_s_end ? 1 : 0);
                     it.seg = t_seg0 + t_s;
                     it.w_once = t_once;
                     it.k0 = t_k0;
@@ -547,8 +584,8 @@ struct ItemWalk {
                 }
                 have_tile = false;
             }
-            if (sj < s_units) {  // next unit of the shared expert: (tile, k chunk, segment pair)
-                const int tc = sj / pairs_s, q = sj - tc * pairs_s;
+            if (sj < s_units) {  // next unit of the shared expert: (tile, k chunk, segment)
+                const int tc = sj / nseg_s, q = sj - tc * nseg_s;
                 const int tile = tc / a.shared_ksplit, chunk = tc - tile * a.shared_ksplit;
                 t_k0 = chunk * a.shared_kchunk;
                 t_k1 = min(a.K[1], t_k0 + a.shared_kchunk);
@@ -561,10 +598,9 @@ struct ItemWalk {
                 t_seg0 = 0;
                 t_n = a.T;
                 t_seg_rows = a.shared_seg;
-                t_s = a.shared_paired ? 2 * q : q;
-                t_s0 = t_s;
-                t_s_end = a.shared_paired ? min(nseg_s, 2 * q + 2) : q + 1;
-                t_once = pairs_s <= 1;
+                t_s = q;
+                t_s_end = q + 1;
+                t_once = nseg_s <= 1;
                 sj += gridDim.x;
                 have_tile = true;
                 continue;
@@ -580,10 +616,10 @@ struct ItemWalk {
                     return false;
                 }
                 if (a.round_robin) {
-                    // one (pair, tile, k chunk) item
+                    // one (segment, tile, k chunk) item
                     const int chunk = lo % a.routed_ksplit;
                     const int tile = (lo / a.routed_ksplit) % ntiles;
-                    g_nseg = (sg.n + FF_SEG - 1) / FF_SEG;
+                    g_nseg = (sg.n + a.seg_rows - 1) / a.seg_rows;
                     t_u0 = tile * max_units;
                     t_h = min(max_units, R0 - t_u0);
                     t_grp = 0;
@@ -591,11 +627,10 @@ struct ItemWalk {
                     t_row0 = sg.row0;
                     t_seg0 = sg.first_seg;
                     t_n = sg.n;
-                    t_seg_rows = FF_SEG;
+                    t_seg_rows = a.seg_rows;
                     t_s = sidx - sg.first_seg;
-                    t_s0 = t_s;
-                    t_s_end = min(g_nseg, t_s + 2);
-                    t_once = g_nseg <= 2;
+                    t_s_end = t_s + 1;
+                    t_once = g_nseg <= 1;
                     t_k0 = chunk * a.routed_kchunk;
                     t_k1 = min(a.K[0], t_k0 + a.routed_kchunk);
                     t_out_off = chunk * a.routed_part_stride;
@@ -613,7 +648,7 @@ struct ItemWalk {
             }
             if (!group_loaded) {
                 sg = a.seg[fs];
-                g_nseg = (sg.n + FF_SEG - 1) / FF_SEG;
+                g_nseg = (sg.n + a.seg_rows - 1) / a.seg_rows;
                 g_u_end = fs == fs_hi ? u_hi : R0;
                 group_loaded = true;
             }
@@ -625,11 +660,10 @@ struct ItemWalk {
                 t_row0 = sg.row0;
                 t_seg0 = sg.first_seg;
                 t_n = sg.n;
-                t_seg_rows = FF_SEG;
+                t_seg_rows = a.seg_rows;
                 t_s = 0;
-                t_s0 = 0;
                 t_s_end = g_nseg;
-                t_once = g_nseg <= 2;
+                t_once = g_nseg <= 1;
                 t_k0 = 0;
                 t_k1 = a.K[0];
                 t_out_off = 0;
@@ -667,22 +701,57 @@ struct XRingWalk {
 
 __device__ __forceinline__ int pieces16(int n) { return (n + 15) >> 4; }
 
+// One output value of an epilogue thread: h = silu(g) * u (GATED) or the plain sum, as bf16.
 template <bool GATED>
-__device__ __forceinline__ void epilogue_store8(const uint32_t *g, const uint32_t *u,
-                                                __nv_bfloat16 *dst)
+__device__ __forceinline__ __nv_bfloat16 epilogue_value(uint32_t g, uint32_t u)
 {
-    uint32_t o[4];
+    float v = __uint_as_float(g);
+    if (GATED)
+        v = silu_f(v) * __uint_as_float(u);
+    return __float2bfloat16_rn(v);
+}
+
+// Epilogue transposition.  An epilogue thread owns one output feature (its TMEM lane) and
+// holds that feature's values for 16 consecutive tokens, but the outputs are token-major
+// (features contiguous).  Two-byte stores of single values cost a fifth of the whole pass at
+// large token counts, so the warp first exchanges values with three rounds of shuffles
+// (lane distances 1, 2, 4): afterwards every lane holds, for two of the 16 tokens, eight
+// consecutive features as one 16-byte vector.
+//   in:  w[c]  bf16 bits (low half) of this lane's feature for token c, c = 0..15
+//   out: v[i]  features 8*(lane>>3) .. +7 of token  tok[i],  i = 0, 1
+__device__ __forceinline__ void transpose_16x32(const uint32_t (&w)[16], int lane, uint4 (&v)[2],
+                                                int (&tok)[2])
+{
+    const bool b1 = lane & 1, b2 = lane & 2, b4 = lane & 4;
+    // distance 1: pairs of features; even lanes keep tokens 0-7, odd lanes tokens 8-15
+    uint32_t p[8];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        float a = __uint_as_float(g[2 * j]), b = __uint_as_float(g[2 * j + 1]);
-        if (GATED) {
-            a = silu_f(a) * __uint_as_float(u[2 * j]);
-            b = silu_f(b) * __uint_as_float(u[2 * j + 1]);
-        }
-        __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
-        o[j] = *reinterpret_cast<uint32_t *>(&p);
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t keep = b1 ? w[8 + i] : w[i];
+        const uint32_t send = b1 ? w[i] : w[8 + i];
+        const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
+        p[i] = b1 ? (recv | (keep << 16)) : (keep | (recv << 16));
     }
-    *reinterpret_cast<uint4 *>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+    // distance 2: four features; the lane of the lower pair keeps the first four of its tokens
+    uint32_t q0[4], q1[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t keep = b2 ? p[4 + i] : p[i];
+        const uint32_t send = b2 ? p[i] : p[4 + i];
+        const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 2);
+        q0[i] = b2 ? recv : keep;
+        q1[i] = b2 ? keep : recv;
+    }
+    // distance 4: eight features, two tokens
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const uint32_t k0 = b4 ? q0[2 + i] : q0[i], k1 = b4 ? q1[2 + i] : q1[i];
+        const uint32_t s0 = b4 ? q0[i] : q0[2 + i], s1 = b4 ? q1[i] : q1[2 + i];
+        const uint32_t r0 = __shfl_xor_sync(0xffffffffu, s0, 4);
+        const uint32_t r1 = __shfl_xor_sync(0xffffffffu, s1, 4);
+        v[i] = b4 ? make_uint4(r0, r1, k0, k1) : make_uint4(k0, k1, r0, r1);
+        tok[i] = (b1 ? 8 : 0) + (b2 ? 4 : 0) + (b4 ? 2 : 0) + i;
+    }
 }
 
 // GATED: W_gate and W_up tiles -> h = silu(g) * u.   !GATED: W_down tiles -> y.
@@ -690,8 +759,7 @@ template <bool GATED>
 __global__ void __launch_bounds__(FF_THREADS, 1)
 ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
 {
-    constexpr int ACC_COLS = 256;      // TMEM columns per accumulator buffer
-    constexpr int NW = GATED ? 2 : 1;  // weight matrices stacked in one N operand
+    constexpr int NW = GATED ? 2 : 1;  // weight matrices per tile (gate and up: one block each)
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * FF_MAX_W_SLOTS + 2 * FF_X_ENTRIES + 4 + 2 * FF_CLAIMS];
@@ -701,8 +769,12 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
 
     const int NS = args.n_w_slots;
     const int kb = args.kboxes;
-    // token ring first: an MMA reads 128 token rows from an entry that may hold fewer, and
-    // the excess of the last entry then falls into the weight ring instead of past the end
+    // TMEM: a set of accumulators is two blocks (gate and up, or two blocks of 128 down rows) of
+    // acc_block columns each; two sets of 2 x 128 columns, or one set of 2 x 256
+    const int acc_sets = args.acc_sets;
+    const uint32_t acc_block = acc_sets == 2 ? 128u : 256u;
+    // token ring first (an MMA reads exactly the rows of its entry, rounded up to 16; a weight
+    // block is read as 128 rows, which for a shorter tile ends inside the slot's capacity)
     const uint32_t ring_x = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle needs 1 KB alignment
     const uint32_t ring_w = ring_x + (uint32_t)args.x_units * FF_X_UNIT;
     const uint32_t bar0 = smem_u32(bars);
@@ -773,8 +845,6 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                     griddep_launch();  // after the wait: dependents may rely on the plan
                     launched = true;
                 }
-                if (it.role == 2)
-                    continue;  // rides on the tile loaded for the first of its pair
                 const int K = it.k1;
                 const uint32_t tile_bytes = (uint32_t)it.h * 128u;
                 const int wrow = it.expert * args.rows[0] + it.f0;  // expert = 0 for the shared kind
@@ -824,7 +894,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             // segment's rows are fetched once its progress counter says they are complete
             ItemWalk walk(args, claims, false, true, false, !GATED);
             XRingWalk ring(args.x_units);
-            int seen[2] = {-1, -1};  // (group, segment) keys last found complete
+            int seen = -1;  // (group kind, segment) key last found complete
             const uint64_t pol_keep = l2_policy_evict_last();
             int released = 0;          // entries known to have been consumed
             int v_cur = 0, v_rel = 0;  // virtual unit positions: issued up to / free up to
@@ -832,73 +902,62 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             bool ok = true;
             Item it;
             while (ok && walk.next(it)) {
-                // a pair alternates its two segments' entries, k step by k step
-                Item it2 = it;
-                const int nsub = it.role == 1 ? 2 : 1;
-                if (nsub == 2 && !walk.next(it2))
-                    break;  // cannot happen: a first is always followed by its second
                 const int K = it.k1;
                 if (!GATED) {
-                    for (int sub = 0; ok && sub < nsub; ++sub) {
-                        const Item &cur = sub ? it2 : it;
-                        const int key = (cur.grp << 30) | cur.seg;
-                        if (key == seen[0] || key == seen[1])
-                            continue;
+                    const int key = (it.grp << 30) | it.seg;
+                    if (key != seen) {
                         // every epilogue warp of the gate/up pass counts the 16-column units
                         // of h it has finished for the segment
-                        ok = counter_wait(args.done[cur.grp] + cur.seg, args.K[cur.grp] >> 2, abortp,
+                        ok = counter_wait(args.done[it.grp] + it.seg, args.K[it.grp] >> 2, abortp,
                                           args.status);
-                        seen[sub] = key;
+                        seen = key;
+                        if (!ok)
+                            break;
+                        // rows written through the generic proxy, read below by the async proxy
+                        asm volatile("fence.proxy.async.global;" ::: "memory");
+                    }
+                }
+                const int pieces = pieces16(it.n);
+                const int m = pieces * kb;
+                for (int k0 = it.k0; ok && k0 < K; k0 += 64 * kb) {
+                    const int nbox = min(kb, (K - k0 + 63) >> 6);
+                    const int j = ring.count;
+                    int pad;
+                    const int at = ring.place(m, pad);
+                    const int v_start = v_cur + pad, v_end = v_start + m;
+                    // the entry's units (and its barrier pair) must have been released:
+                    // everything before the oldest entry still in use is free, the
+                    // padding in front of it included
+                    while (released < j &&
+                           (j - released >= FF_X_ENTRIES || v_end - v_rel > args.x_units)) {
+                        const int r = released % FF_X_ENTRIES;
+                        if (!mbar_wait(x_empty(r), (uint32_t)(released / FF_X_ENTRIES) & 1u, abortp,
+                                       args.status)) {
+                            ok = false;
+                            break;
+                        }
+                        ++released;
+                        v_rel = released < j ? v_start_of[released % FF_X_ENTRIES] : v_start;
                     }
                     if (!ok)
                         break;
-                    // rows written through the generic proxy, read below by the async proxy
-                    asm volatile("fence.proxy.async.global;" ::: "memory");
-                }
-                for (int k0 = it.k0; ok && k0 < K; k0 += 64 * kb) {
-                    const int nbox = min(kb, (K - k0 + 63) >> 6);
-                    for (int sub = 0; sub < nsub; ++sub) {
-                        const Item &cur = sub ? it2 : it;
-                        const int pieces = pieces16(cur.n);
-                        const int m = pieces * kb;
-                        const int j = ring.count;
-                        int pad;
-                        const int at = ring.place(m, pad);
-                        const int v_start = v_cur + pad, v_end = v_start + m;
-                        // the entry's units (and its barrier pair) must have been released:
-                        // everything before the oldest entry still in use is free, the
-                        // padding in front of it included
-                        while (released < j &&
-                               (j - released >= FF_X_ENTRIES || v_end - v_rel > args.x_units)) {
-                            const int r = released % FF_X_ENTRIES;
-                            if (!mbar_wait(x_empty(r), (uint32_t)(released / FF_X_ENTRIES) & 1u, abortp,
-                                           args.status)) {
-                                ok = false;
-                                break;
-                            }
-                            ++released;
-                            v_rel = released < j ? v_start_of[released % FF_X_ENTRIES] : v_start;
-                        }
-                        if (!ok)
-                            break;
-                        const int e = j % FF_X_ENTRIES;
-                        v_start_of[e] = v_start;
-                        v_cur = v_end;
-                        const uint32_t base = ring_x + (uint32_t)at * FF_X_UNIT;
-                        mbar_expect_tx(x_full(e), (uint32_t)(nbox * pieces) * FF_X_UNIT);
-                        for (int b = 0; b < nbox; ++b) {
-                            // the entry's rows as boxes of 128, 64, 32 and 16 rows
-                            uint32_t dst = base + (uint32_t)(b * pieces) * FF_X_UNIT;
-                            int row = cur.row0, rem = pieces << 4;
-                            while (rem > 0) {
-                                const int hi = rem >= 128 ? 0 : (rem >= 64 ? 1 : (rem >= 32 ? 2 : 3));
-                                const int bh = 128 >> hi;
-                                tma_load_2d_hint(dst, &maps.x[it.grp][hi], x_full(e), k0 + 64 * b, row,
-                                                 pol_keep);
-                                dst += (uint32_t)bh * 128u;
-                                row += bh;
-                                rem -= bh;
-                            }
+                    const int e = j % FF_X_ENTRIES;
+                    v_start_of[e] = v_start;
+                    v_cur = v_end;
+                    const uint32_t base = ring_x + (uint32_t)at * FF_X_UNIT;
+                    mbar_expect_tx(x_full(e), (uint32_t)(nbox * pieces) * FF_X_UNIT);
+                    for (int b = 0; b < nbox; ++b) {
+                        // the entry's rows as boxes of 128, 64, 32 and 16 rows
+                        uint32_t dst = base + (uint32_t)(b * pieces) * FF_X_UNIT;
+                        int row = it.row0, rem = pieces << 4;
+                        while (rem > 0) {
+                            const int hi = rem >= 128 ? 0 : (rem >= 64 ? 1 : (rem >= 32 ? 2 : 3));
+                            const int bh = 128 >> hi;
+                            tma_load_2d_hint(dst, &maps.x[it.grp][hi], x_full(e), k0 + 64 * b, row,
+                                             pol_keep);
+                            dst += (uint32_t)bh * 128u;
+                            row += bh;
+                            rem -= bh;
                         }
                     }
                 }
@@ -919,73 +978,57 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             int n_items = 0;
             Item it;
             while (ok && walk.next(it)) {
-                Item it2 = it;
-                const int nsub = it.role == 1 ? 2 : 1;
-                if (nsub == 2 && !walk.next(it2))
-                    break;  // cannot happen: a first is always followed by its second
-                // accumulator buffers: each is waited for right before its first instruction, so
-                // that the first segment of a pair starts while the epilogue still drains the
-                // other buffer
-                int buf[2];
-                uint32_t acc_par[2];
-                bool acc_ready[2] = {false, false};
-                for (int sub = 0; sub < nsub; ++sub) {
-                    buf[sub] = n_items & 1;
-                    acc_par[sub] = ((uint32_t)(n_items >> 1) & 1u) ^ 1u;
-                    ++n_items;
-                }
+                // the accumulator set is waited for right before the item's first instruction, so
+                // that its operands are already being fetched while the epilogue drains the set
+                const int set = n_items % acc_sets;
+                const uint32_t acc_par = ((uint32_t)(n_items / acc_sets) & 1u) ^ 1u;
+                ++n_items;
+                bool acc_ready = false;
+                const uint32_t d0 = tmem_base + (uint32_t)set * 2u * acc_block;
                 const uint32_t tile_bytes = (uint32_t)it.h * 128u;
-                const uint32_t idesc = umma_idesc_bf16(NW * it.h);
+                const int pieces = pieces16(it.n);
+                const uint32_t idesc = umma_idesc_bf16(pieces << 4);  // M = 128, N = token rows
+                // weight blocks of the tile: gate and up, or the 128-row halves of a down tile
+                const int nblk = GATED ? 2 : (it.h + 127) >> 7;
+                // descriptor steps in 16-byte units: to the next block, to the next k box
+                const uint32_t blk16 = (GATED ? tile_bytes : 128u * 128u) >> 4;
+                const uint64_t w_box16 = (uint64_t)((NW * tile_bytes) >> 4);
+                const uint64_t x_box16 = (uint64_t)((pieces * FF_X_UNIT) >> 4);
                 const int K = it.k1;
                 for (int k0 = it.k0; ok && k0 < K; k0 += 64 * kb) {
                     const int nbox = min(kb, (K - k0 + 63) >> 6);
-                    // the weight slot is multiplied with one or two segments' token entries
-                    uint32_t xbase[2], xpar[2];
-                    int xe[2], pieces[2];
-                    for (int sub = 0; sub < nsub; ++sub) {
-                        pieces[sub] = pieces16(sub ? it2.n : it.n);
-                        const int j = ring.count;
-                        int pad;
-                        const int at = ring.place(pieces[sub] * kb, pad);
-                        xe[sub] = j % FF_X_ENTRIES;
-                        xpar[sub] = (uint32_t)(j / FF_X_ENTRIES) & 1u;
-                        xbase[sub] = ring_x + (uint32_t)at * FF_X_UNIT;
-                    }
-                    if (!mbar_wait(w_full(sw), pw, abortp, args.status)) {
+                    const int j = ring.count;
+                    int pad;
+                    const int at = ring.place(pieces * kb, pad);
+                    const int xe = j % FF_X_ENTRIES;
+                    const uint32_t xpar = (uint32_t)(j / FF_X_ENTRIES) & 1u;
+                    const uint32_t xbase = ring_x + (uint32_t)at * FF_X_UNIT;
+                    if (!mbar_wait(w_full(sw), pw, abortp, args.status) ||
+                        !mbar_wait(x_full(xe), xpar, abortp, args.status)) {
                         ok = false;
                         break;
                     }
-                    const uint32_t wbase = ring_w + sw * args.w_slot_bytes;
-                    for (int sub = 0; sub < nsub; ++sub) {
-                        // the second segment's rows may still be landing while the first
-                        // segment's instructions run
-                        if (!mbar_wait(x_full(xe[sub]), xpar[sub], abortp, args.status)) {
+                    tc_fence_after();
+                    if (!acc_ready) {
+                        if (!mbar_wait(acc_empty(set), acc_par, abortp, args.status)) {
                             ok = false;
                             break;
                         }
                         tc_fence_after();
-                        if (!acc_ready[sub]) {
-                            if (!mbar_wait(acc_empty(buf[sub]), acc_par[sub], abortp, args.status)) {
-                                ok = false;
-                                break;
-                            }
-                            tc_fence_after();
-                            acc_ready[sub] = true;
-                        }
-                        const uint32_t d0 = tmem_base + (uint32_t)(buf[sub] * ACC_COLS);
-                        for (int b = 0; b < nbox; ++b) {
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const uint32_t accum = ((k0 - it.k0) | b | q) != 0 ? 1u : 0u;
-                                umma_bf16(d0,
-                                          umma_desc_sw128(xbase[sub] + (uint32_t)(b * pieces[sub]) * FF_X_UNIT + q * 32),
-                                          umma_desc_sw128(wbase + b * NW * tile_bytes + q * 32), idesc, accum);
-                            }
-                        }
-                        umma_commit(x_empty(xe[sub]));
+                        acc_ready = true;
                     }
-                    if (!ok)
-                        break;
+                    uint64_t w_desc = umma_desc_sw128(ring_w + sw * args.w_slot_bytes);
+                    uint64_t x_desc = umma_desc_sw128(xbase);
+                    for (int b = 0; b < nbox; ++b) {
+                        const uint32_t accum = ((k0 - it.k0) | b) != 0 ? 1u : 0u;
+                        if (nblk == 2)
+                            issue_k_box<2>(d0, acc_block, w_desc, blk16, x_desc, idesc, accum);
+                        else
+                            issue_k_box<1>(d0, acc_block, w_desc, blk16, x_desc, idesc, accum);
+                        w_desc += w_box16;
+                        x_desc += x_box16;
+                    }
+                    umma_commit(x_empty(xe));
                     umma_commit(w_empty(sw));  // reusable once these MMAs have read it
                     if (++sw == NS) {
                         sw = 0;
@@ -993,8 +1036,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                     }
                 }
                 if (ok)
-                    for (int sub = 0; sub < nsub; ++sub)
-                        umma_commit(acc_full(buf[sub]));  // accumulators complete
+                    umma_commit(acc_full(set));  // accumulators complete
             }
             if (!walk.synced)
                 walk.sync(true);
@@ -1012,43 +1054,62 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
             // executed by every lane
             if (!walk.next(it))
                 break;
-            const int buf = n_items & 1;
-            const uint32_t acc_phase = (uint32_t)(n_items >> 1) & 1u;
+            const int set = n_items % acc_sets;
+            const uint32_t acc_phase = (uint32_t)(n_items / acc_sets) & 1u;
             ++n_items;
             // every lane waits; the vote makes the decision uniform and reconverges the warp
             // for the warp-collective tcgen05.ld below
-            const bool ready = mbar_wait(acc_full(buf), acc_phase, abortp, args.status);
+            const bool ready = mbar_wait(acc_full(set), acc_phase, abortp, args.status);
             if (!__all_sync(0xffffffffu, ready))
                 break;
             tc_fence_after();
-            if (quarter * 32 < it.n) {
-                const int trow = quarter * 32 + lane;  // token row of this thread
-                const bool row_ok = trow < it.n;
-                __nv_bfloat16 *out =
-                    args.out[it.grp] + it.out_off + (size_t)(it.row0 + trow) * args.out_ld[it.grp] + it.f0;
-                const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * ACC_COLS);
-                // two register buffers: the TMEM load of the next 16 columns is in flight while
-                // the current 16 are converted and stored
+            // a thread owns one weight row (output feature) of a block and walks the tokens
+            const int nblk = GATED ? 1 : (it.h + 127) >> 7;  // gate and up are read together
+            const int ld = args.out_ld[it.grp];
+            const int npad = pieces16(it.n) << 4;
+            for (int m = 0; m < nblk; ++m) {
+                const int rows_blk = GATED ? it.h : min(128, it.h - 128 * m);
+                if (quarter * 32 >= rows_blk)
+                    break;  // this warp's lanes lie beyond the tile (uniform)
+                // after the transposition this lane stores features 8 * (lane >> 3) .. + 7 of
+                // the warp's 32 (tiles are multiples of 16 features: all eight exist or none)
+                const int fgrp = quarter * 32 + 8 * (lane >> 3);
+                const bool grp_ok = fgrp < rows_blk;
+                __nv_bfloat16 *out = args.out[it.grp] + it.out_off + (size_t)it.row0 * ld + it.f0 +
+                                     128 * m + fgrp;
+                const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) +
+                                    (uint32_t)set * 2u * acc_block + (uint32_t)m * acc_block;
+                // two register buffers: the TMEM load of the next 16 tokens is in flight while
+                // the current 16 are converted, transposed and stored
                 uint32_t g[2][16], u[2][16];
                 tmem_ld16(t0, g[0]);
                 if (GATED)
-                    tmem_ld16(t0 + it.h, u[0]);
+                    tmem_ld16(t0 + acc_block, u[0]);
 #pragma unroll 1
-                for (int c = 0; c < it.h; c += 32) {
+                for (int c = 0; c < npad; c += 32) {
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
                         const int cc = c + 16 * half;
-                        if (cc < it.h) {
+                        if (cc < npad) {
                             tmem_ld_wait();
-                            if (cc + 16 < it.h) {
+                            if (cc + 16 < npad) {
                                 tmem_ld16(t0 + cc + 16, g[half ^ 1]);
                                 if (GATED)
-                                    tmem_ld16(t0 + it.h + cc + 16, u[half ^ 1]);
+                                    tmem_ld16(t0 + acc_block + cc + 16, u[half ^ 1]);
                             }
-                            if (row_ok) {
-                                epilogue_store8<GATED>(g[half], u[half], out + cc);
-                                epilogue_store8<GATED>(g[half] + 8, u[half] + 8, out + cc + 8);
+                            uint32_t w[16];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                const __nv_bfloat16 val = epilogue_value<GATED>(g[half][i], u[half][i]);
+                                w[i] = (uint32_t)__bfloat16_as_ushort(val);
                             }
+                            uint4 v[2];
+                            int tok[2];
+                            transpose_16x32(w, lane, v, tok);
+#pragma unroll
+                            for (int i = 0; i < 2; ++i)
+                                if (grp_ok && cc + tok[i] < it.n)
+                                    *reinterpret_cast<uint4 *>(out + (size_t)(cc + tok[i]) * ld) = v[i];
                         }
                     }
                 }
@@ -1058,7 +1119,7 @@ ffn_fused_kernel(const FfnArgs args, const __grid_constant__ FfnMaps maps)
                 asm volatile("fence.proxy.async.global;" ::: "memory");
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(acc_empty(buf));
+                mbar_arrive(acc_empty(set));
                 if (GATED) {
                     // publish: this warp's part of the tile is in h (a releasing reduction: the
                     // warp does not wait for its stores to become visible, the counter does)
@@ -1286,13 +1347,34 @@ static double expected_active_experts(int E, int k, int T)
 
 static int ffn_grid() { return sm_count(); }
 
-// Up to 128 tokens no group of the layer has more than one 128-row segment, so no two token
-// entries must be resident together and the token ring can be 32 KB, which leaves room for a
-// third weight slot (worth 3-4 % of the layer) -- provided the entries stay within half of the
-// ring, i.e. 64 rows: always so up to 64 tokens; between 65 and 128 tokens only while the
-// routed groups are expected to be small (a larger group still works, its rows are then not
-// fetched ahead), and the shared expert's rows are then cut into two 64-row segments that run
-// as single items.
+// Segment size of a call (the N limit of its tensor-core instructions).  Groups in the hundreds
+// of rows want the contraction geometry: segments of 256 rows, so that a weight tile is fetched
+// once per 256 tokens and the instruction runs at its full rate.  Small groups want the
+// streaming geometry (segments of 128 rows, 64 KB weight slots, double-buffered accumulators).
+// The host never sees the routing result, so it decides on the expected rows per group -- and on
+// the shared expert, whose group is all T tokens: where its weights are a large part of the
+// layer's, every extra segment is another pass over them through L2.
+int ffn_segment_rows(const moe_config_t &c, int T)
+{
+    const int force = geometry_override();
+    if (force >= 0)
+        return force == 1 ? FF_SEG_WIDE : FF_SEG;
+    if (T <= FF_SEG)
+        return FF_SEG;
+    // measured cross-over: about 112 expected rows per group (most groups then exceed one
+    // 128-row segment), or a shared expert several times an expert's size
+    const double rows_per_group = (double)T * c.top_k / expected_active_experts(c.n_experts, c.top_k, T);
+    if (rows_per_group > 0.875 * FF_SEG)
+        return FF_SEG_WIDE;
+    return c.shared_inter >= 6 * c.inter ? FF_SEG_WIDE : FF_SEG;
+}
+
+// Up to 128 tokens no group of the layer has more than one 128-row segment and the token ring
+// can be 32 KB, which leaves room for a third weight slot (worth 3-4 % of the layer) --
+// provided the entries stay within half of the ring, i.e. 64 rows: always so up to 64 tokens;
+// between 65 and 128 tokens only while the routed groups are expected to be small (a larger
+// group still works, its rows are then not fetched ahead), and the shared expert's rows are
+// then cut into two 64-row segments.
 static bool small_token_ring(const moe_config_t &c, int T)
 {
     if (T <= FF_SEG / 2)
@@ -1306,26 +1388,27 @@ static bool small_token_ring(const moe_config_t &c, int T)
 // Token rows per segment of the shared expert (see small_token_ring).
 static int shared_segment_rows(const moe_config_t &c, int T)
 {
-    return (T > FF_SEG / 2 && small_token_ring(c, T)) ? FF_SEG / 2 : FF_SEG;
+    if (T > FF_SEG / 2 && small_token_ring(c, T))
+        return FF_SEG / 2;
+    return ffn_segment_rows(c, T);
 }
 
 // Number of tiles the shared expert's rows are cut into.  The shared expert's work units are
-// (tile, segment pair); a unit should cost about the expected per-CTA share of the whole pass
-// (or less), with the tile height within [min_tile, max_tile] rows: a tensor-core
-// instruction costs the same for any tile height, so tiles below 128 stacked rows (the N
-// operand) would make the pass issue-bound.
+// (tile, k chunk, segment); a unit should cost about the expected per-CTA share of the whole
+// pass (or less), with the tile height within [min_tile, max_tile] rows (a weight block
+// costs the same instruction time whether it holds 16 rows or 128).
 static int shared_tile_count(const moe_config_t &c, int T, int rows_routed, int rows_shared,
                              int K_routed, int K_shared, int ksplit, int min_tile, int max_tile,
                              int grid)
 {
-    const int nseg_s = (T + shared_segment_rows(c, T) - 1) / shared_segment_rows(c, T);
-    const int pairs_s = T > FF_SEG ? (nseg_s + 1) / 2 : nseg_s;
+    const int seg_s = shared_segment_rows(c, T), seg_r = ffn_segment_rows(c, T);
+    const int nseg_s = (T + seg_s - 1) / seg_s;
     const int units = rows_shared >> 4;
     const double k_ratio = (double)K_shared / K_routed;  // cost of a shared row unit per segment
     const double n_act = expected_active_experts(c.n_experts, c.top_k, T);
-    const double segs_r = n_act * ceil((double)T * c.top_k / n_act / FF_SEG);
+    const double segs_r = n_act * ceil((double)T * c.top_k / n_act / seg_r);
     const double total = units * k_ratio * nseg_s + segs_r * (rows_routed >> 4);
-    int tu = (int)ceil(total / grid / (k_ratio / ksplit * nseg_s / pairs_s));
+    int tu = (int)ceil(total / grid / (k_ratio / ksplit));
     if (tu < (min_tile >> 4))
         tu = min_tile >> 4;
     if (tu > (max_tile >> 4))
@@ -1333,17 +1416,19 @@ static int shared_tile_count(const moe_config_t &c, int T, int rows_routed, int 
     return (units + tu - 1) / tu;
 }
 
-// Ring geometry: two k boxes per weight slot (64 KB for a full tile: every row is fetched in
-// 256 contiguous bytes, which both HBM and L2 serve markedly faster than 128).  The token
-// ring holds two entries of the largest possible segment while no group can exceed 64 rows,
-// three 128-row entries otherwise (a pair of segments needs two at once).
+// Ring geometry.  Streaming: two k boxes per weight slot (64 KB for a full tile: every row is
+// fetched in 256 contiguous bytes, which both HBM and L2 serve markedly faster than 128); the
+// token ring holds two entries of the largest possible segment while no group can exceed 64
+// rows (32 KB, three weight slots), three 128-row entries otherwise (96 KB, two slots).
+// Contraction: one k box per slot and per entry, three 256-row entries (96 KB), four slots.
 static void ffn_geometry(const moe_config_t &c, int T, FfnArgs &a)
 {
-    a.kboxes = 2;
-    a.w_slot_bytes = 256 * 128 * a.kboxes;  // a full tile: 256 stacked rows per k box
-    // entries never wrap, so two entries that must be resident together (a pair of segments:
-    // 32 KB + up to 32 KB) need a ring of three of them wherever the first may sit
-    const int x_ring_bytes = small_token_ring(c, T) ? 32 * 1024 : 96 * 1024;
+    a.seg_rows = ffn_segment_rows(c, T);
+    const bool wide = a.seg_rows > FF_SEG;
+    a.kboxes = wide ? 1 : 2;
+    a.acc_sets = wide ? 1 : 2;
+    a.w_slot_bytes = 256 * 128 * a.kboxes;  // a full tile: 256 rows per k box
+    const int x_ring_bytes = (!wide && small_token_ring(c, T)) ? 32 * 1024 : 96 * 1024;
     a.x_units = x_ring_bytes / FF_X_UNIT;
     const int avail = FF_SMEM_LIMIT - 1024 - 512;  // alignment slack, static shared memory
     int ns = (avail - x_ring_bytes) / a.w_slot_bytes;
@@ -1352,17 +1437,16 @@ static void ffn_geometry(const moe_config_t &c, int T, FfnArgs &a)
     a.n_w_slots = ns;
     a.wait_us = (int)(FF_WAIT_NS / 1000ull);
     a.shared_seg = shared_segment_rows(c, T);
-    a.shared_paired = T > FF_SEG ? 1 : 0;
 }
 
 // Range mode keeps every CTA alone on "its" groups, perfectly levelled.  It loses when
-//  - a range is shorter than a few tiles: its two ends are partial tiles, and a tile of any
-//    height costs K/16 tensor-core instructions, so short ranges turn issue-bound;
+//  - a range is shorter than a few tiles: its two ends are partial tiles, and a weight block
+//    costs K/16 tensor-core instructions whatever its height, so short ranges turn issue-bound;
 //  - the token rows of `grid` groups do not fit in L2 beside the weight stream (large T): every
 //    tile would fetch its group's rows from HBM again.
 // Then, and when there are so many tiles per CTA that the last wave hardly matters, the routed
-// work is dealt round-robin as (pair, tile) items: full tiles only, and the CTAs work on a few
-// groups at a time.
+// work is dealt round-robin as (segment, tile) items: full tiles only, and the CTAs work on a
+// few groups at a time.
 static bool use_round_robin(const moe_config_t &c, int T, int rows_routed, int K_routed, int max_tile,
                             int grid)
 {
@@ -1371,8 +1455,8 @@ static bool use_round_robin(const moe_config_t &c, int T, int rows_routed, int K
         return force == 1;
     const double n_act = expected_active_experts(c.n_experts, c.top_k, T);
     const double rows_per_group = (double)T * c.top_k / n_act;
-    const double pairs = n_act * ceil(ceil(rows_per_group / FF_SEG) / 2.0);
-    const double tiles_per_cta = pairs * ((rows_routed + max_tile - 1) / max_tile) / grid;
+    const double segs = n_act * ceil(rows_per_group / ffn_segment_rows(c, T));
+    const double tiles_per_cta = segs * ((rows_routed + max_tile - 1) / max_tile) / grid;
     const double token_bytes = rows_per_group * K_routed * 2.0 * grid;
     return tiles_per_cta < 3.0 || tiles_per_cta >= 12.0 || token_bytes > 200.0 * 1024 * 1024;
 }
@@ -1393,8 +1477,6 @@ static cudaError_t launch_ffn(FfnArgs &a, const FfnMaps &maps, cudaStream_t s)
             return e;
         configured.mark(dev);
     }
-    // the 128-row read of the last token entry may run 16 KB past the token ring: the weight
-    // ring behind it is always larger than that
     const size_t smem = (size_t)a.x_units * FF_X_UNIT + (size_t)a.n_w_slots * a.w_slot_bytes + 1024;
     if (a.n_w_slots < 2 || smem > FF_SMEM_LIMIT - 512)
         return cudaErrorInvalidConfiguration;
@@ -1460,17 +1542,17 @@ cudaError_t launch_ffn_gateup(const moe_config_t &c, const moe_weights_t &w, con
 static int split_chunk(int K, int parts) { return ((K + parts - 1) / parts + 127) / 128 * 128; }
 static int split_parts(int K, int parts) { return (K + split_chunk(K, parts) - 1) / split_chunk(K, parts); }
 
-// Expected number of (segment pair, tile) items of the routed down pass; never decreases
-// with T.
+// Expected number of (segment, tile) items of the routed down pass (counted with the wide
+// segments, so that it never decreases with T).
 static double routed_down_items(const moe_config_t &c, int T)
 {
     const double n_act = expected_active_experts(c.n_experts, c.top_k, T);
     const double rows_per_group = (double)T * c.top_k / n_act;
-    return ceil(n_act) * ceil(ceil(rows_per_group / FF_SEG) / 2.0) * ((c.hidden + 255) / 256);
+    return ceil(n_act) * ceil(rows_per_group / FF_SEG_WIDE) * ((c.hidden + 255) / 256);
 }
 
 // k chunks of the routed groups' down projection.  While the pass has fewer than about three
-// (pair, tile) items per CTA -- few tokens, or few experts with long reductions -- some SMs
+// (segment, tile) items per CTA -- few tokens, or few experts with long reductions -- some SMs
 // have no weight stream to pull and one SM cannot pull a tile faster than a fraction of what
 // HBM delivers, so the reduction is cut; each chunk writes its own plane of y and the combine
 // adds the planes.  (Fewer than three items per CTA also means the pass deals single items.)

@@ -50,7 +50,7 @@ __device__ void block_exclusive_scan(int *vals, int *tmp, int n, int *total)
 }
 
 // Segment plan from per-expert counts and offsets held in shared memory: one entry per
-// segment of SEG_TOKENS rows of every activated expert, in ascending expert order.  All
+// segment of plan.seg_rows rows of every activated expert, in ascending expert order.  All
 // threads of the block must call it; scan/tmp/total are shared scratch.
 __device__ void build_plan(const int *cnt_sh, const int *off_sh, int *scan, int *tmp, int *total,
                            int E, int32_t *status, PlanView plan)
@@ -58,7 +58,7 @@ __device__ void build_plan(const int *cnt_sh, const int *off_sh, int *scan, int 
     const int tid = threadIdx.x;
     const int cnt = tid < E ? cnt_sh[tid] : 0;
     const int row0 = tid < E ? off_sh[tid] : 0;
-    const int nseg = (cnt + SEG_TOKENS - 1) / SEG_TOKENS;
+    const int nseg = (cnt + plan.seg_rows - 1) / plan.seg_rows;
     __syncthreads();
     if (tid < MOE_MAX_EXPERTS)
         scan[tid] = nseg;
@@ -78,23 +78,17 @@ __device__ void build_plan(const int *cnt_sh, const int *off_sh, int *scan, int 
     }
     if (tid == 0)
         plan.header[0] = *total;
-    // pairs: segments 2q and 2q+1 of a group
+    // the item list: one entry per segment, carrying its group
     const int first = nseg > 0 ? scan[tid] : 0;
-    const int npair = (nseg + 1) >> 1;
-    __syncthreads();
-    if (tid < MOE_MAX_EXPERTS)
-        scan[tid] = npair;
-    __syncthreads();
-    block_exclusive_scan(scan, tmp, E, total);
-    for (int q = 0; q < npair; ++q) {
+    for (int q = 0; q < nseg; ++q) {
         PairEntry pe;
         pe.expert = tid;
         pe.row0 = row0;
         pe.n = cnt;
         pe.first_seg = first;
-        pe.seg = first + 2 * q;
+        pe.seg = first + q;
         pe.pad[0] = pe.pad[1] = pe.pad[2] = 0;
-        plan.pairs[scan[tid] + q] = pe;
+        plan.pairs[first + q] = pe;
     }
     if (tid == 0) {
         plan.header[1] = *total;

@@ -1,17 +1,20 @@
 """Model of how the FFN kernels hand out the routed work (CPU only).
 
 `ffn_fused_kernel` lays the weight rows of all routed groups end to end -- one position =
-16 weight rows of one group for one of its 128-row segments -- and its CTAs claim chunks
-[lo, hi) of positions from a grid-wide counter.  A chunk's two ends are mapped to (group, row
-unit) and moved down to a tile boundary of that group; inside its chunk a CTA processes whole
-tiles, each for all segments of the group.  This test replays that rule for random groups
-and random claim sizes and checks what the kernels rely on: every (group, tile) is processed
-by exactly one chunk, whatever the claim sizes, and in round-robin mode every
-(segment pair, tile, k chunk) item exactly once.
+16 weight rows of one group for one of its segments (128 or 256 token rows, fixed per call) --
+and its CTAs claim chunks [lo, hi) of positions from a grid-wide counter.  A chunk's two ends
+are mapped to (group, row unit) and moved down to a tile boundary of that group; inside its
+chunk a CTA processes whole tiles, each for all segments of the group.  This test replays that
+rule for random groups and random claim sizes and checks what the kernels rely on: every
+(group, tile) is processed by exactly one chunk, whatever the claim sizes, and in round-robin
+mode every (segment, tile, k chunk) item exactly once.
+
+It restates `ItemWalk::boundary`, the range walk of `ItemWalk::next` and `ItemWalk::claim`
+(csrc/ffn_fused.cu) in Python: a change to those functions has to be made here as well.
 """
 import random
 
-SEG = 128
+SEG = 128   # set per test: the segment size of the call
 
 
 def n_segments(rows):
@@ -48,8 +51,10 @@ def tiles_of_chunk(lo, hi, groups, first_seg, R0, max_units):
 
 
 def test_every_tile_is_claimed_exactly_once_in_range_mode():
+    global SEG
     rng = random.Random(7)
-    for _ in range(300):
+    for trial in range(300):
+        SEG = 128 if trial % 2 else 256
         R0 = rng.choice([88, 160, 128, 37])            # 16-row units of weight rows per group
         max_units = rng.choice([8, 16])
         groups = [rng.choice([1, 5, 16, 100, 128, 129, 200, 257, 400]) for _ in range(rng.randint(1, 12))]
@@ -72,14 +77,14 @@ def test_every_tile_is_claimed_exactly_once_in_range_mode():
         assert len(seen) == len(groups) * R0, "row units missing"
 
 
-def test_round_robin_items_cover_every_pair_tile_and_k_chunk_once():
+def test_round_robin_items_cover_every_segment_tile_and_k_chunk_once():
     rng = random.Random(8)
     for _ in range(200):
         grid = rng.choice([4, 148])
         ntiles = rng.randint(1, 23)
         ksplit = rng.randint(1, 8)
-        npairs = rng.randint(1, 40)
-        P = npairs * ntiles * ksplit
+        nsegs = rng.randint(1, 40)
+        P = nsegs * ntiles * ksplit
         items = []
         counter = 0
         ctas = list(range(grid))

@@ -133,6 +133,17 @@ def test_row_permutation_equivariance():
     assert torch.equal(out_p, out[p])
 
 
+@pytest.mark.parametrize("wide", ["0", "1"])
+def test_layer_parity_in_both_ring_geometries(wide):
+    """The FFN kernels run with segments of up to 128 token rows (two k boxes per weight slot,
+    two sets of accumulators) or of up to 256 (one k box, one set); MOE_FF_WIDE (a test hook
+    read once per process) forces one of the two on every call, also where the host would
+    choose the other: the scheduling cases and a few small shapes in a child process each."""
+    _run_child({"MOE_FF_WIDE": wide},
+               "scheduling_mode_case or (small_shapes and (qwen-like or dense-contrast or "
+               "ksplit-routed or ragged or e24-33tok or dsv3-like-zipf))")
+
+
 def test_layer_parity_with_plain_stream_ordering():
     """MOE_NO_PDL=1 (read once per process) launches every kernel with plain stream ordering:
     the kernels then run one after the other and every progress counter is complete when its

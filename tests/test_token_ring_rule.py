@@ -3,10 +3,13 @@
 The token-operand ring of `ffn_fused_kernel` holds entries of 2 KB units that never wrap: an
 entry that does not fit before the end of the ring starts at unit 0, and the producer may place
 entry j once everything before the oldest entry still in use is free.  The MMA side consumes
-the entries of one k step together (one entry, or two for a pair of segments).  This test
-replays that rule over random item sequences: the geometries the host chooses (48 units with
-pairs of segments, 16 units without, i.e. up to 128 tokens) never stall and never overlap live entries, and a ring
-of exactly two full entries with pairs does stall -- which is why the host refuses it.
+one entry per k step.  This test replays that rule over random item sequences: the geometries
+the host chooses -- 48 units for segments of up to 16 units (128 rows at two k boxes per entry,
+or 256 rows at one), 16 units for batches of up to 128 tokens -- never stall and never overlap
+live entries.
+
+It restates `XRingWalk::place` and the release loop of the token producer (csrc/ffn_fused.cu)
+in Python: a change to those has to be made here as well.
 """
 import random
 
@@ -68,42 +71,34 @@ def replay(units, steps):
     return "ok"
 
 
-def random_steps(rng, max_pieces, pairs):
-    """Items as the kernels produce them: a full first segment (16 units at two k boxes per
-    slot) with any second segment, or a single segment; sizes are even (two k boxes)."""
+def random_steps(rng, max_units, even):
+    """Items as the kernels produce them: one entry per k step, all k steps of an item of the
+    same size (even in the streaming geometry: two k boxes per entry)."""
     steps = []
     for _ in range(rng.randint(1, 8)):
         k_steps = rng.randint(1, 6)
-        if pairs and rng.random() < 0.5:
-            steps += [[2 * max_pieces, 2 * rng.randint(1, max_pieces)]] * k_steps
-        else:
-            steps += [[2 * rng.randint(1, max_pieces)]] * k_steps
+        m = rng.randint(1, max_units // 2) * 2 if even else rng.randint(1, max_units)
+        steps += [[m]] * k_steps
     return steps
 
 
-def test_ring_of_three_full_entries_never_stalls_with_pairs():
+def test_large_ring_never_stalls():
+    """96 KB: entries of up to 16 units (a full segment in either geometry)."""
     rng = random.Random(1)
     for _ in range(4000):
-        assert replay(48, random_steps(rng, 8, True)) == "ok"
+        assert replay(48, random_steps(rng, 16, True)) == "ok"
+    for _ in range(4000):
+        assert replay(48, random_steps(rng, 16, False)) == "ok"
 
 
-def test_small_ring_never_stalls_without_pairs():
-    """Up to 128 tokens no group has two segments: single entries only, of up to half the ring
-    (the shared expert's 64-row segments, groups of up to 64 rows) or, for a routed group of up
-    to 128 rows, of the whole ring."""
+def test_small_ring_never_stalls():
+    """Up to 128 tokens: entries of up to half the ring (the shared expert's 64-row segments,
+    groups of up to 64 rows) or, for a routed group of up to 128 rows, of the whole ring."""
     rng = random.Random(2)
     for _ in range(4000):
-        assert replay(16, random_steps(rng, 4, False)) == "ok"
+        assert replay(16, random_steps(rng, 8, True)) == "ok"
     for _ in range(4000):
-        assert replay(16, random_steps(rng, 8, False)) == "ok"
-
-
-def test_ring_of_two_full_entries_can_stall_with_pairs():
-    # a 16-unit entry that sits at unit 10 leaves no room for its 14-unit partner
-    assert replay(32, [[10]] * 4 + [[16, 14]] * 2) == "stall"
-    rng = random.Random(3)
-    outcomes = {replay(32, random_steps(rng, 8, True)) for _ in range(2000)}
-    assert "overlap" not in outcomes and "stall" in outcomes
+        assert replay(16, random_steps(rng, 16, True)) == "ok"
 
 
 def test_entries_in_flight_are_bounded_by_the_barrier_pairs():
