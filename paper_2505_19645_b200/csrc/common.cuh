@@ -314,8 +314,16 @@ __device__ __forceinline__ void status_region_init(int32_t *status)
     }
 }
 
-// g * sigmoid(g) with the fast exponential and division (the result is rounded to bf16)
-__device__ __forceinline__ float silu_f(float g) { return __fdividef(g, 1.0f + __expf(-g)); }
+// g * sigmoid(g) = g * (0.5 + 0.5 * tanh(g / 2)) with the hardware tanh: one special-function
+// operation per value instead of two (exponential and reciprocal); its relative error, about
+// 2^-11, is a quarter of the bf16 rounding the result goes through
+__device__ __forceinline__ float silu_f(float g)
+{
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * g));
+    const float half_g = 0.5f * g;
+    return fmaf(half_g, t, half_g);
+}
 
 #endif  // __CUDACC__
 
