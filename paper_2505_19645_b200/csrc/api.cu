@@ -381,9 +381,23 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
     } arm;
     const PlanView plan = plan_view(base, L, ffn_segment_rows(*cfg, T));
     int32_t *status = reinterpret_cast<int32_t *>(base + L.status);
-    MOE_STAGE(MOE_STAGE_ROUTER_LOGITS,
-              launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s,
-                                   plan.done_shared, max_shared_segments(T), status));
+    if (router_logits_tc_applies(*cfg, T)) {
+        const bool probe_ = g_probe_armed && g_probe.stage == MOE_STAGE_ROUTER_LOGITS;
+        if (probe_ && cudaEventRecord(g_probe.start, s) != cudaSuccess)
+            return MOE_ERR_CUDA;
+        if (launch_router_logits_tc(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr,
+                                    reinterpret_cast<__nv_bfloat16 *>(base + L.rl_planes),
+                                    reinterpret_cast<float *>(base + L.rl_partial), s,
+                                    plan.done_shared, max_shared_segments(T), status,
+                                    &launches) != cudaSuccess)
+            return MOE_ERR_CUDA;
+        if (probe_ && cudaEventRecord(g_probe.stop, s) != cudaSuccess)
+            return MOE_ERR_CUDA;
+    } else {
+        MOE_STAGE(MOE_STAGE_ROUTER_LOGITS,
+                  launch_router_logits(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr, s,
+                                       plan.done_shared, max_shared_segments(T), status));
+    }
     // the grouping kernel also writes the FFN segment plan (one launch fewer); for a small
     // batch it selects the experts and gathers the token rows as well (three fewer)
     const bool small = route_group_small_applies(*cfg, T);

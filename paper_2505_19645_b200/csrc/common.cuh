@@ -89,6 +89,8 @@ struct Workspace {
     size_t h_shared;      // bf16 [T, I_s]
     size_t y;             // bf16 [A, H]      expert outputs, sorted order
     size_t y_shared;      // bf16 [shared_down_parts, T, H]: partial sums per k chunk
+    size_t rl_planes;     // bf16 [3, R, H]: router rows as three bf16 terms (large batches only)
+    size_t rl_partial;    // f32 [k chunks, T, R]: partial logits (large batches only)
     size_t total;
     // every region in layout order (offset, bytes in use); the bytes between two regions --
     // the rounding up to 256 and a guard of WS_GUARD_BYTES -- belong to no kernel
@@ -126,6 +128,11 @@ constexpr int ROUTED_SPLIT_MAX_PARTS = 8;
 int routed_down_parts(const moe_config_t &c, int T);
 size_t routed_split_max_rows(const moe_config_t &c, int T);
 
+// regions of the tensor-core router-logit path (0 bytes where a call does not use it)
+bool router_logits_tc_applies(const moe_config_t &c, int T);
+size_t router_tc_plane_bytes(const moe_config_t &c, int T);
+size_t router_tc_partial_bytes(const moe_config_t &c, int T);
+
 inline Workspace workspace_layout(const moe_config_t &c, int T)
 {
     Workspace w{};
@@ -155,6 +162,8 @@ inline Workspace workspace_layout(const moe_config_t &c, int T)
     const size_t y_rows = A > A_split ? A : A_split;
     w.y = cut.take(y_rows * H * 2);
     w.y_shared = cut.take((size_t)T * H * 2 * shared_down_parts(c));
+    w.rl_planes = cut.take(router_tc_plane_bytes(c, T));
+    w.rl_partial = cut.take(router_tc_partial_bytes(c, T));
     w.total = cut.off;
     return w;
 }
@@ -169,6 +178,13 @@ cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
                                  const __nv_bfloat16 *x, int T, float *logits,
                                  float *shared_scale, cudaStream_t s, int32_t *zero = nullptr,
                                  int zero_n = 0, int32_t *status = nullptr);
+// The same on tcgen05 for large batches (router_logits_tc.cu): three launches (split of the fp32
+// rows into bf16 planes, the contraction, the sum of its k chunks); planes / partial are the
+// workspace regions of router_tc_plane_bytes / router_tc_partial_bytes.
+cudaError_t launch_router_logits_tc(const moe_config_t &c, const moe_weights_t &w,
+                                    const __nv_bfloat16 *x, int T, float *logits, float *shared_scale,
+                                    __nv_bfloat16 *planes, float *partial, cudaStream_t s,
+                                    int32_t *zero, int zero_n, int32_t *status, int *launches);
 cudaError_t launch_route_topk(const moe_config_t &c, const float *logits, int T, int32_t *idx,
                               float *wts, cudaStream_t s);
 cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int32_t *counts,
