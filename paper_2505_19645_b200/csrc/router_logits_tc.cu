@@ -13,8 +13,9 @@
 //   reduce  sums the S partial planes in a fixed order, adds the bias, applies the sigmoid
 // The reduction over H is cut into S chunks so that about one CTA per SM has work even when
 // there are only a dozen token tiles; the partial planes are summed in chunk order, so the
-// logits do not depend on timing.  Used from 512 tokens on, where the mma.sync kernel of
-// router_logits.cu (which splits the rows on the fly for every token tile) takes 60-300 us.
+// logits do not depend on timing.  Used for large batches (router_logits_tc_applies), where the
+// mma.sync kernel of router_logits.cu, which splits the rows on the fly for every token tile,
+// takes 60-300 us.
 #include <string.h>
 
 #include <mutex>
@@ -32,9 +33,11 @@ constexpr int RT_B_BYTES = RT_TOKENS * 128;
 constexpr int RT_MAX_SPLIT = 16;
 constexpr int RT_SMEM = RT_A_SLOTS * RT_A_BYTES + RT_B_SLOTS * RT_B_BYTES + 1024;
 
+// From about 128 K logits on the mma.sync kernel takes longer than the three launches here
+// (measured: 256 experts from 512 tokens, 64 experts from 2048 tokens).
 bool router_logits_tc_applies(const moe_config_t &c, int T)
 {
-    return T >= 512 && c.n_experts >= 32 && c.hidden >= 512;
+    return T >= 512 && (long long)T * c.n_experts >= 128 * 1024 && c.hidden >= 512;
 }
 
 static int router_rows(const moe_config_t &c)

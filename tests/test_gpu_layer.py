@@ -39,10 +39,10 @@ def test_tiny_config_full_parity():
     ("e8-warp-dup", 128, 8, 2, 256, 0, 0, 1, 0, 3, 4, None),           # 30 assignments on 8 experts
     ("e24-32tok", 256, 24, 16, 128, 128, 0, 0, 1, 8, 3, None),         # 32 tokens x top-16: 512 assignments
     ("e24-33tok", 256, 24, 16, 128, 128, 0, 0, 1, 11, 2, None),        # one token more: the long chain
-    # from 512 tokens on the router logits run on tcgen05 (three bf16 planes, k chunks)
-    ("tc-logits-gate", 512, 60, 4, 128, 128, 0, 0, 1, 130, 3, None),   # 520 tokens, gate row (R = 61)
+    # large batches (T * E >= 128 K): router logits on tcgen05 (three bf16 planes, k chunks)
+    ("tc-logits-gate", 512, 60, 4, 128, 128, 0, 0, 1, 550, 3, None),   # 2200 tokens, gate row (R = 61)
     ("tc-logits-2pairs", 512, 300, 4, 64, 0, 1, 1, 0, 200, 2, 1.0),    # two pairs of row blocks, bias
-    ("tc-logits-ragged", 544, 130, 2, 64, 64, 0, 1, 1, 171, 2, None),  # 513 tokens, half k box, R = 131
+    ("tc-logits-ragged", 544, 130, 2, 64, 64, 0, 1, 1, 337, 2, None),  # 1011 tokens, half k box, R = 131
 ])
 def test_layer_parity_small_shapes(name, H, E, k, I, Is, score, renorm, sgate, B, gamma, zipf):
     shape = wl.small_shape(name, H, E, k, I, Is, score, renorm, sgate)
