@@ -292,13 +292,16 @@ def sweep_points(config):
     return pts, [(B, g) for B, g in EXTRA_POINTS.get(config, []) if B * (g + 1) not in have]
 
 
-def run_sweep(config, shape, runner, peaks, per_pass, device):
+def run_sweep(config, shape, runner, peaks, per_pass, device, grid=None):
     """Every (B, gamma) point of the config's grid (plus the extra token counts).  A point is
     visited in three passes over the grid -- at the large shapes the part sits at its power cap,
     where the SM clock steps on the time scale of one visit -- and reported by the MEDIAN of all
     its samples; the lowest of the three pass medians and the fastest sample are kept beside it
     under their own keys."""
-    grid, extra = sweep_points(config)
+    if grid is None:
+        grid, extra = sweep_points(config)
+    else:
+        extra = []
     samples = {}
     for _ in range(3):
         for (Bi, gi) in grid + extra:
@@ -308,7 +311,6 @@ def run_sweep(config, shape, runner, peaks, per_pass, device):
             samples.setdefault((Bi, gi), []).append(ms)
     E, k = shape.n_experts, shape.top_k
     t_thres = token_threshold(E, k)
-    gs = wl.GRIDS[config][1]
     base = {}
     rows = []
     for (Bi, gi) in grid + extra:
@@ -325,7 +327,7 @@ def run_sweep(config, shape, runner, peaks, per_pass, device):
         roof, bound = roof_ms(shape, Ti, na, peaks["hbm_gbs"], peaks["bf16_tflops"])
         roof_sus, _ = roof_ms(shape, Ti, na, peaks["hbm_gbs"], peaks["bf16_tflops_sustained"])
         roof_nom, _ = roof_ms(shape, Ti, na, NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS)
-        ratio = med / base[Bi] if (Bi in base and gs[0] == 0 and (Bi, gi) in grid) else None
+        ratio = med / base[Bi] if (Bi in base and (Bi, gi) in grid) else None
         rows.append({
             "B": Bi, "gamma": gi, "T": Ti, "extra": (Bi, gi) in extra,
             "us": round(med * 1e3, 2), "us_best_pass": round(best_pass * 1e3, 2),
@@ -667,26 +669,11 @@ def main():
         held["w"] = None
         torch.cuda.empty_cache()
         if args.sweeps == "config" and args.grid == "sparsity":
-            Bs, gs = wl.SPARSITY_BATCHES, wl.SPARSITY_GAMMAS
-            runner.prepare(max(Bs) * (max(gs) + 1))
-            rows = []
-            for Bi in Bs:
-                base_ms = None
-                for gi in gs:
-                    Ti = Bi * (gi + 1)
-                    xi = wl.make_tokens(shape, Ti, wl.point_seed(args.config, Bi, gi), device)
-                    ms = []
-                    for _ in range(3):
-                        ms += runner.time_steps(xi, Bi, gi, per_pass, 3)[0]
-                    med = statistics.median(ms)
-                    base_ms = med if gi == 0 else base_ms
-                    na = runner.n_active(xi, Bi, gi)
-                    rf, _ = roof_ms(shape, Ti, na, peaks["hbm_gbs"], peaks["bf16_tflops"])
-                    rows.append({"B": Bi, "gamma": gi, "T": Ti, "us": round(med * 1e3, 2),
-                                 "n_active": na, "roof_frac": round(rf / med, 4),
-                                 "ratio_vs_gamma0": round(med / base_ms, 4)})
-            sweeps["sparsity:" + shape.name] = {"config": args.config, "shape": shape.as_dict(),
-                                                "rows": rows}
+            grid = [(Bi, gi) for Bi in wl.SPARSITY_BATCHES for gi in wl.SPARSITY_GAMMAS]
+            runner.prepare(max(Bi * (gi + 1) for Bi, gi in grid))
+            key = "sparsity:" + shape.name
+            sweeps[key] = run_sweep(args.config, shape, runner, peaks, per_pass, device, grid=grid)
+            sweeps[key]["zipf"] = args.zipf
     clocks = sampler.stop()
 
     # ---- CPU oracle beside it (rank 0, N = 1) -----------------------------------------
