@@ -163,6 +163,16 @@ struct ClaimRing {
 // tile).  Round-robin mode: a chunk is one (segment, tile, k chunk) item; consecutive items are
 // the tiles of one segment, which then run on many CTAs at once and share the segment's token
 // rows in L2.
+// Rows per segment of a group of n rows cut into nseg segments: equal shares rounded up to the
+// 16-row unit of the token boxes (never more than the segment limit, since nseg = ceil(n /
+// limit)).  Equal shares instead of "full segments and a remainder": the instruction time
+// follows the rows of a segment with a floor of about 64 rows, so 320 rows cost less as
+// 160 + 160 than as 256 + 64.
+__device__ __forceinline__ int balanced_segment_rows(int n, int nseg)
+{
+    return (((n + nseg - 1) / nseg) + 15) & ~15;
+}
+
 struct ItemWalk {
     const FfnArgs &a;
     const ClaimRing &ring;
@@ -363,7 +373,7 @@ struct ItemWalk {
                 t_row0 = 0;
                 t_seg0 = 0;
                 t_n = a.T;
-                t_seg_rows = a.shared_seg;
+                t_seg_rows = balanced_segment_rows(a.T, nseg_s);
                 t_s = q;
                 t_s_end = q + 1;
                 t_once = nseg_s <= 1;
@@ -393,7 +403,7 @@ struct ItemWalk {
                     t_row0 = sg.row0;
                     t_seg0 = sg.first_seg;
                     t_n = sg.n;
-                    t_seg_rows = a.seg_rows;
+                    t_seg_rows = balanced_segment_rows(sg.n, g_nseg);
                     t_s = sidx - sg.first_seg;
                     t_s_end = t_s + 1;
                     t_once = g_nseg <= 1;
@@ -426,7 +436,7 @@ struct ItemWalk {
                 t_row0 = sg.row0;
                 t_seg0 = sg.first_seg;
                 t_n = sg.n;
-                t_seg_rows = a.seg_rows;
+                t_seg_rows = balanced_segment_rows(sg.n, g_nseg);
                 t_s = 0;
                 t_s_end = g_nseg;
                 t_once = g_nseg <= 1;
