@@ -218,6 +218,31 @@ moe_status_t run_ffn(const moe_config_t &c, const moe_weights_t &w, const __nv_b
 
 using namespace moe;
 
+// Copies of the layer's intermediates for the caller (moe_debug_out_t), enqueued behind the layer.
+static moe_status_t copy_debug_out(const moe_config_t &c, int T, const moe_debug_out_t *dbg,
+                                   const char *base, const Workspace &L, cudaStream_t s)
+{
+    if (!dbg)
+        return MOE_OK;
+    const size_t A = (size_t)T * c.top_k, E = c.n_experts;
+    struct Copy {
+        void *dst;
+        size_t src;
+        size_t bytes;
+    } copies[] = {
+        {dbg->logits, L.logits, (size_t)T * E * 4}, {dbg->topk_idx, L.topk_idx, A * 4},
+        {dbg->topk_w, L.topk_w, A * 4},             {dbg->counts, L.counts, E * 4},
+        {dbg->offsets, L.offsets, (E + 1) * 4},     {dbg->perm, L.perm, A * 4},
+        {dbg->inv_perm, L.inv_perm, A * 4},         {dbg->active, L.active, E * 4},
+        {dbg->n_active, L.n_active, 4},
+    };
+    for (const Copy &cp : copies)
+        if (cp.dst && cudaMemcpyAsync(cp.dst, base + cp.src, cp.bytes, cudaMemcpyDeviceToDevice, s) !=
+                          cudaSuccess)
+            return MOE_ERR_CUDA;
+    return MOE_OK;
+}
+
 extern "C" {
 
 size_t moe_workspace_bytes(const moe_config_t *cfg, int32_t max_tokens)
@@ -359,6 +384,20 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char *base = static_cast<char *>(ws);
     const __nv_bfloat16 *xb = static_cast<const __nv_bfloat16 *>(x);
+    if (layer_small_applies(*cfg, T)) {
+        // a handful of tokens: the whole layer is one launch (its time is recorded as the
+        // gate/up stage's, the stage that dominates it)
+        const bool probe_ = g_probe.stage == MOE_STAGE_GATE_UP;
+        if (probe_ && cudaEventRecord(g_probe.start, s) != cudaSuccess)
+            return MOE_ERR_CUDA;
+        if (launch_layer_small(*cfg, *w, xb, T, static_cast<__nv_bfloat16 *>(out), base, L, s) !=
+            cudaSuccess)
+            return MOE_ERR_CUDA;
+        if (probe_ && cudaEventRecord(g_probe.stop, s) != cudaSuccess)
+            return MOE_ERR_CUDA;
+        g_last_launches = 1;
+        return copy_debug_out(*cfg, T, dbg, base, L, s);
+    }
     float *logits = reinterpret_cast<float *>(base + L.logits);
     int32_t *topk_idx = reinterpret_cast<int32_t *>(base + L.topk_idx);
     float *topk_w = reinterpret_cast<float *>(base + L.topk_w);
@@ -423,25 +462,7 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
                              static_cast<__nv_bfloat16 *>(out), s));
     g_last_launches = launches;
 
-    if (dbg) {
-        const size_t A = (size_t)T * cfg->top_k, E = cfg->n_experts;
-        struct Copy {
-            void *dst;
-            const void *src;
-            size_t bytes;
-        } copies[] = {
-            {dbg->logits, logits, (size_t)T * E * 4}, {dbg->topk_idx, topk_idx, A * 4},
-            {dbg->topk_w, topk_w, A * 4},             {dbg->counts, counts, E * 4},
-            {dbg->offsets, offsets, (E + 1) * 4},     {dbg->perm, perm, A * 4},
-            {dbg->inv_perm, inv_perm, A * 4},         {dbg->active, active, E * 4},
-            {dbg->n_active, n_active, 4},
-        };
-        for (const Copy &cp : copies)
-            if (cp.dst && cudaMemcpyAsync(cp.dst, cp.src, cp.bytes, cudaMemcpyDeviceToDevice, s) !=
-                              cudaSuccess)
-                return MOE_ERR_CUDA;
-    }
-    return MOE_OK;
+    return copy_debug_out(*cfg, T, dbg, base, L, s);
 }
 
 moe_status_t moe_check(void *ws, void *stream)

@@ -64,7 +64,7 @@ __host__ __device__ inline int max_segments(int E, int A) { return E + A / SEG_T
 // ---------------------------------------------------------------------------------------
 // Workspace layout (every region 256-byte aligned).
 // ---------------------------------------------------------------------------------------
-constexpr int WS_MAX_REGIONS = 24;
+constexpr int WS_MAX_REGIONS = 32;
 constexpr size_t WS_GUARD_BYTES = 256;  // never written: lets a test detect a store that strays
 
 struct Workspace {
@@ -91,6 +91,8 @@ struct Workspace {
     size_t y_shared;      // bf16 [shared_down_parts, T, H]: partial sums per k chunk
     size_t rl_planes;     // bf16 [3, R, H]: router rows as three bf16 terms (large batches only)
     size_t rl_partial;    // f32 [k chunks, T, R]: partial logits (large batches only)
+    size_t small_logit_part;  // f32 [E + 1, column chunks, 4]: partial logits of the one-launch layer
+    size_t small_y_part;      // f32 [chunks, rows, H]: partial expert outputs of the one-launch layer
     size_t total;
     // every region in layout order (offset, bytes in use); the bytes between two regions --
     // the rounding up to 256 and a guard of WS_GUARD_BYTES -- belong to no kernel
@@ -133,6 +135,11 @@ bool router_logits_tc_applies(const moe_config_t &c, int T);
 size_t router_tc_plane_bytes(const moe_config_t &c, int T);
 size_t router_tc_partial_bytes(const moe_config_t &c, int T);
 
+// the whole layer in one launch for a handful of tokens (layer_small.cu); its two regions
+bool layer_small_applies(const moe_config_t &c, int T);
+size_t layer_small_logit_part_bytes(const moe_config_t &c);
+size_t layer_small_y_part_bytes(const moe_config_t &c, int T);
+
 inline Workspace workspace_layout(const moe_config_t &c, int T)
 {
     Workspace w{};
@@ -164,6 +171,8 @@ inline Workspace workspace_layout(const moe_config_t &c, int T)
     w.y_shared = cut.take((size_t)T * H * 2 * shared_down_parts(c));
     w.rl_planes = cut.take(router_tc_plane_bytes(c, T));
     w.rl_partial = cut.take(router_tc_partial_bytes(c, T));
+    w.small_logit_part = cut.take(layer_small_logit_part_bytes(c));
+    w.small_y_part = cut.take(layer_small_y_part_bytes(c, T));
     w.total = cut.off;
     return w;
 }
@@ -227,6 +236,13 @@ cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, int ro
                            const __nv_bfloat16 *shared_y, int shared_parts,
                            const float *shared_scale, int T, __nv_bfloat16 *out, cudaStream_t s);
 
+// Router logits, top-k, grouping, expert FFNs, shared expert and combine of at most four tokens
+// in one cooperative launch; uses the regions status, logits .. inv_perm, h, h_shared,
+// small_logit_part and small_y_part of `L` in `ws`.
+cudaError_t launch_layer_small(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x,
+                               int T, __nv_bfloat16 *out, char *ws, const Workspace &L,
+                               cudaStream_t s);
+
 int sm_count();
 bool pdl_enabled();  // programmatic dependent launch between the layer's kernels
 // Test hook, read once per process from MOE_FF_RR: 0 / 1 forces the FFN kernels to deal the
@@ -234,6 +250,9 @@ bool pdl_enabled();  // programmatic dependent launch between the layer's kernel
 int schedule_override();
 // The same for the ring geometry, from MOE_FF_WIDE: 0 / 1 forces segments of 128 / 256 rows.
 int geometry_override();
+// From MOE_SMALL_FUSED: 0 keeps calls of a few tokens on the chain of kernels every other call
+// uses, -1 (unset) lets them take the one-launch kernel.
+int small_layer_override();
 // Token rows per segment of the routed groups for a call with T tokens: 128 or 256 (the plan and
 // the FFN kernels of one call must agree on it).
 int ffn_segment_rows(const moe_config_t &c, int T);

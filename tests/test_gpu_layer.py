@@ -92,6 +92,57 @@ def test_layer_parity_in_both_scheduling_modes(mode):
     _run_child({"MOE_FF_RR": mode}, "scheduling_mode_case")
 
 
+# One to four tokens with at most 32 assignments take the one-launch kernel (logits, routing,
+# expert FFNs and combine behind grid barriers); MOE_SMALL_FUSED=0 keeps them on the kernel chain.
+FEW_TOKEN_CASES = [
+    ("few-qwen", 512, 60, 4, 352, 1408, 0, 0, 1, 1, 0, None),        # T = 1, shared expert + gate
+    ("few-qwen-4", 512, 60, 4, 352, 1408, 0, 0, 1, 2, 1, None),      # T = 4
+    ("few-dsv3", 1024, 256, 8, 256, 256, 1, 1, 0, 1, 3, None),       # sigmoid, 32 assignments
+    ("few-dsv3-3", 1024, 256, 8, 256, 256, 1, 1, 0, 3, 0, 1.0),      # T = 3, skewed, bias
+    ("few-mixtral", 512, 8, 2, 1792, 0, 0, 1, 0, 1, 2, None),        # no shared expert
+    ("few-dup", 256, 4, 2, 384, 256, 0, 1, 0, 2, 1, None),           # 8 assignments on 4 experts: up to 4 rows each
+    ("few-dense", 128, 4, 4, 256, 0, 0, 1, 0, 4, 0, None),           # k = E: every group has all 4 rows
+    ("few-ragged", 160, 6, 3, 224, 96, 0, 1, 0, 1, 1, None),         # rows shorter than a lane step
+    ("few-chunks", 384, 8, 2, 4352, 2176, 0, 0, 1, 3, 0, None),      # down projection in 3 and 2 column chunks, ragged last
+    ("few-e512", 256, 512, 16, 128, 128, 1, 1, 0, 1, 1, 1.0),        # the expert limit, top-16 x 2 tokens
+    ("few-k16-3tok", 256, 24, 16, 128, 128, 0, 0, 1, 3, 0, None),    # 48 assignments: stays on the chain
+    ("few-dense-contrast", 256, 1, 1, 3072, 3072, 0, 0, 1, 2, 1, None),  # E = k = 1
+]
+
+
+@pytest.mark.parametrize("name,H,E,k,I,Is,score,renorm,sgate,B,gamma,zipf", FEW_TOKEN_CASES)
+def test_few_token_case(name, H, E, k, I, Is, score, renorm, sgate, B, gamma, zipf):
+    shape = wl.small_shape(name, H, E, k, I, Is, score, renorm, sgate)
+    w = wl.make_weights(shape, 500 + E, "cuda", zipf_s=zipf)
+    T = B * (gamma + 1)
+    x = wl.make_tokens(shape, T, 600 + T, "cuda")
+    check_layer_against_oracle(shape, w, x, B, gamma)
+
+
+def test_few_tokens_take_one_launch():
+    from paper_2505_19645_b200 import api
+
+    shape = wl.small_shape("few-launch", 512, 60, 4, 352, 1408, 0, 0, 1)
+    w = wl.make_weights(shape, 21, "cuda")
+    x = wl.make_tokens(shape, 4, 22, "cuda")
+    out_a, dbg_a = run_gpu_layer(shape, w, x, 2, 1)
+    assert api.moe_last_launch_count() == 1
+    out_b, dbg_b = run_gpu_layer(shape, w, x, 4, 0)
+    assert torch.equal(out_a, out_b)
+    for key in dbg_a:
+        np.testing.assert_array_equal(dbg_a[key], dbg_b[key])
+    # the fifth token moves the call to the kernel chain
+    x5 = wl.make_tokens(shape, 5, 23, "cuda")
+    run_gpu_layer(shape, w, x5, 5, 0)
+    assert api.moe_last_launch_count() > 1
+
+
+def test_kernel_chain_on_the_same_few_tokens():
+    """The same cases with the one-launch kernel switched off (a test hook read once per
+    process, hence the child process)."""
+    _run_child({"MOE_SMALL_FUSED": "0"}, "test_few_token_case")
+
+
 def test_layer_depends_on_token_count_only_and_is_deterministic():
     """layer(B, gamma) == layer(B*(gamma+1), 0) bit for bit; two runs and a run on another
     stream give identical routing, grouping and outputs."""

@@ -112,7 +112,7 @@ def test_workspace_regions_are_disjoint_aligned_and_guarded():
         cfg = api.make_config(wl.CONFIGS[name])
         total = api.moe_workspace_bytes(cfg, T)
         regions = api.workspace_regions(cfg, T)
-        assert len(regions) == 22
+        assert len(regions) == 24
         end = 0
         for i, (off, n) in enumerate(regions):
             assert off % 256 == 0
@@ -120,6 +120,18 @@ def test_workspace_regions_are_disjoint_aligned_and_guarded():
             end = off + n
         assert end + 256 <= total
         assert regions[0] == (0, 256)   # the status region leads the workspace
+
+
+def test_workspace_size_never_shrinks_as_tokens_grow():
+    """A workspace sized for max_tokens serves every call with fewer tokens: the layout of a
+    call with T tokens must fit moe_workspace_bytes(T') for every T' >= T (regions that only
+    small or only large calls use must not make the total dip in between)."""
+    from paper_2505_19645_b200 import api
+
+    for name in ("tiny", "qwen1.5-moe-a2.7b", "qwen2-57b-a14b", "mixtral-8x7b", "deepseek-v3"):
+        cfg = api.make_config(wl.CONFIGS[name])
+        sizes = [api.moe_workspace_bytes(cfg, T) for T in list(range(1, 70)) + [127, 128, 129, 511, 512, 513, 2048]]
+        assert all(b >= a for a, b in zip(sizes, sizes[1:])), name
 
 
 def test_per_device_set_up_state_is_kept_per_ordinal(tmp_path):
