@@ -91,8 +91,8 @@ struct Workspace {
     size_t y_shared;      // bf16 [shared_down_parts, T, H]: partial sums per k chunk
     size_t rl_planes;     // bf16 [3, R, H]: router rows as three bf16 terms (large batches only)
     size_t rl_partial;    // f32 [k chunks, T, R]: partial logits (large batches only)
-    size_t small_logit_part;  // f32 [E + 1, column chunks, 4]: partial logits of the one-launch layer
-    size_t small_y_part;      // f32 [chunks, rows, H]: partial expert outputs of the one-launch layer
+    size_t small_logit_part;  // unit counters, then f32 [E + 1, column chunks, 4]: partial logits of the one-launch layer
+    size_t small_h;           // bf16 [rows, padded I] + [T, padded I_s]: SwiGLU intermediates of the one-launch layer
     size_t total;
     // every region in layout order (offset, bytes in use); the bytes between two regions --
     // the rounding up to 256 and a guard of WS_GUARD_BYTES -- belong to no kernel
@@ -138,7 +138,7 @@ size_t router_tc_partial_bytes(const moe_config_t &c, int T);
 // the whole layer in one launch for a handful of tokens (layer_small.cu); its two regions
 bool layer_small_applies(const moe_config_t &c, int T);
 size_t layer_small_logit_part_bytes(const moe_config_t &c);
-size_t layer_small_y_part_bytes(const moe_config_t &c, int T);
+size_t layer_small_h_bytes(const moe_config_t &c, int T);
 
 inline Workspace workspace_layout(const moe_config_t &c, int T)
 {
@@ -172,7 +172,7 @@ inline Workspace workspace_layout(const moe_config_t &c, int T)
     w.rl_planes = cut.take(router_tc_plane_bytes(c, T));
     w.rl_partial = cut.take(router_tc_partial_bytes(c, T));
     w.small_logit_part = cut.take(layer_small_logit_part_bytes(c));
-    w.small_y_part = cut.take(layer_small_y_part_bytes(c, T));
+    w.small_h = cut.take(layer_small_h_bytes(c, T));
     w.total = cut.off;
     return w;
 }
@@ -237,8 +237,8 @@ cudaError_t launch_combine(const moe_config_t &c, const __nv_bfloat16 *y, int ro
                            const float *shared_scale, int T, __nv_bfloat16 *out, cudaStream_t s);
 
 // Router logits, top-k, grouping, expert FFNs, shared expert and combine of at most four tokens
-// in one cooperative launch; uses the regions status, logits .. inv_perm, h, h_shared,
-// small_logit_part and small_y_part of `L` in `ws`.
+// in one cooperative launch; uses the regions status, logits .. inv_perm, small_logit_part and
+// small_h of `L` in `ws`.
 cudaError_t launch_layer_small(const moe_config_t &c, const moe_weights_t &w, const __nv_bfloat16 *x,
                                int T, __nv_bfloat16 *out, char *ws, const Workspace &L,
                                cudaStream_t s);
