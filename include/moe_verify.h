@@ -208,7 +208,14 @@ moe_status_t moe_combine(const moe_config_t *cfg, const void *y, const int32_t *
  * combine adds them in fp32: an expert output then carries up to 8 bf16 roundings instead of
  * one, the shared expert's likewise (its chunk count depends on the shape only).  How many
  * chunks are used depends on T, so a token's low-order bits may differ between batch sizes;
- * the result stays within the layer's stated tolerance at every size. */
+ * the result stays within the layer's stated tolerance at every size.
+ * One to four tokens (with T*top_k <= 32 and a shared expert of moderate size) run as ONE
+ * cooperative launch: partial router logits, then top-k and grouping repeated by every CTA,
+ * then the expert projections on the CUDA cores with the weights streamed once.  There the
+ * SwiGLU intermediate is still rounded to bf16, but the expert outputs stay in fp32 until the
+ * gate-weighted sum, which is rounded once.  Calls that use the same workspace must not overlap
+ * on the GPU (as for every entry point); the device needs cooperative-launch support, else
+ * the call takes the kernel sequence of the larger sizes. */
 moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, const void *x,
                               int32_t B, int32_t gamma, void *out, const moe_debug_out_t *dbg,
                               void *ws, size_t ws_bytes, void *stream);

@@ -41,7 +41,10 @@ constexpr int LS_MAX_ASSIGN = 32;     // T * top_k: one warp sorts the assignmen
 constexpr int LS_MAX_UNITS = 1 + LS_MAX_ASSIGN;  // the shared expert and the activated experts
 constexpr int LS_LOGIT_CHUNK = 1024;  // router-row columns per work item
 constexpr int LS_ROUTE_WARPS = 4;     // warps of every CTA that wait for the logits and do the routing
-constexpr int LS_DOWN_CHUNK = 2048;   // most columns of a down-projection work item
+constexpr int LS_DOWN_CHUNK_MAX = 4096;  // most columns of a down-projection work item ...
+constexpr int LS_DOWN_CHUNK_MIN = 2048;  // ... and the least the host goes down to for more items
+constexpr int LS_DOWN_ITEMS_WANTED = 48; // down-projection items per CTA (three per warp) it aims at
+constexpr size_t LS_SHARED_WORK_MAX = 80u << 20;  // T * I_s * H up to which the kernel is used for T > 1
 constexpr int LS_DOWN_ROWS = 4;       // output features per down-projection work item
 constexpr int LS_SLOT_FLOATS = LS_DOWN_ROWS * LS_MAX_TOKENS;  // partial sums of one such item
 constexpr size_t LS_MAX_SLOT_BYTES = 160u << 10;
@@ -226,18 +229,27 @@ __device__ __forceinline__ void down_item(const __nv_bfloat16 *wd, int ld, int f
 //
 // A 64-bit word: the call's epoch in the high half, a count in the low half.  The workspace need
 // not be initialised and may hold the word of an earlier call (complete or abandoned): whoever
-// adds first finds another epoch there and replaces the word by (epoch, 0) before anybody counts.
+// finds another epoch there replaces the word by (epoch, own count); counts that went to the stale
+// word meanwhile are repeated by their owners.
 __device__ __forceinline__ void tagged_add(unsigned long long *word, uint32_t epoch)
 {
+    // count first: all but the call's first few arrivals find the epoch in place
+    if ((uint32_t)(atomicAdd(word, 1ull) >> 32) == epoch)
+        return;
+    // the add went to a stale word: install (epoch, 1), or count again if somebody else has
+    // installed the epoch meanwhile (adds to the stale word are dropped with it)
     const unsigned long long base = (unsigned long long)epoch << 32;
     unsigned long long seen = *reinterpret_cast<volatile unsigned long long *>(word);
-    while ((uint32_t)(seen >> 32) != epoch) {
-        const unsigned long long prev = atomicCAS(word, seen, base);
+    for (;;) {
+        if ((uint32_t)(seen >> 32) == epoch) {
+            atomicAdd(word, 1ull);
+            return;
+        }
+        const unsigned long long prev = atomicCAS(word, seen, base + 1ull);
         if (prev == seen)
-            break;
+            return;
         seen = prev;
     }
-    atomicAdd(word, 1ull);
 }
 
 // Bounded wait (one thread) until the word reads (epoch, target); acquire.  On giving up raises
@@ -464,11 +476,20 @@ __global__ void __launch_bounds__(LS_THREADS, 1) layer_small_kernel(const SmallA
                     const int t = idx / E, e = idx - t * E;
                     p[u] = a.logit_part + (size_t)e * a.logit_chunks * LS_MAX_TOKENS + t;
                 }
-#pragma unroll 2
-                for (int c = 0; c < a.logit_chunks; ++c)
+                for (int c0 = 0; c0 < a.logit_chunks; c0 += 8) {
+                    float v[8][4];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        z[u] += __ldcg(p[u] + c * LS_MAX_TOKENS);
+                    for (int c = 0; c < 8; ++c)
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            v[c][u] = c0 + c < a.logit_chunks ? __ldcg(p[u] + (c0 + c) * LS_MAX_TOKENS)
+                                                              : 0.f;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            z[u] += v[c][u];
+                }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int idx = idx0 + u * RT;
@@ -764,12 +785,30 @@ __global__ void __launch_bounds__(LS_THREADS, 1) layer_small_kernel(const SmallA
 
 // ---- host -------------------------------------------------------------------------------------
 
-static int down_chunks(int cols) { return (cols + LS_DOWN_CHUNK - 1) / LS_DOWN_CHUNK; }
+// Most columns of a down-projection item for this shape: long items stream best, but a CTA needs
+// a few items per warp to keep all of them busy -- the longest chunk that leaves it
+// LS_DOWN_ITEMS_WANTED items at one token (T = 1: top_k groups), else the shortest.
+static int down_chunk_limit(const moe_config_t &c)
+{
+    const int blocks = (c.hidden / LS_DOWN_ROWS + sm_count() - 1) / sm_count();
+    for (int chunk = LS_DOWN_CHUNK_MAX; chunk > LS_DOWN_CHUNK_MIN; chunk /= 2) {
+        const int uc = (c.shared_inter + chunk - 1) / chunk + c.top_k * ((c.inter + chunk - 1) / chunk);
+        if (uc * blocks >= LS_DOWN_ITEMS_WANTED)
+            return chunk;
+    }
+    return LS_DOWN_CHUNK_MIN;
+}
+
+static int down_chunks(const moe_config_t &c, int cols)
+{
+    const int limit = down_chunk_limit(c);
+    return (cols + limit - 1) / limit;
+}
 
 // columns per chunk: equal shares, rounded up to whole parts of the row walk
-static int down_chunk_cols(int cols)
+static int down_chunk_cols(const moe_config_t &c, int cols)
 {
-    const int n = down_chunks(cols);
+    const int n = down_chunks(c, cols);
     return n == 0 ? 0 : (((cols + n - 1) / n) + 255) & ~255;
 }
 
@@ -779,13 +818,18 @@ static size_t pitch(int cols) { return ((size_t)cols + 63) & ~(size_t)63; }  // 
 static size_t slot_bytes(const moe_config_t &c, int T)
 {
     const size_t blocks = ((size_t)c.hidden / LS_DOWN_ROWS + sm_count() - 1) / sm_count();
-    const size_t uc = (size_t)down_chunks(c.shared_inter) + (size_t)T * c.top_k * down_chunks(c.inter);
+    const size_t uc = (size_t)down_chunks(c, c.shared_inter) + (size_t)T * c.top_k * down_chunks(c, c.inter);
     return uc * blocks * LS_SLOT_FLOATS * sizeof(float);
 }
 
 static bool small_shape(const moe_config_t &c, int T)
 {
-    return T <= LS_MAX_TOKENS && T * c.top_k <= LS_MAX_ASSIGN && slot_bytes(c, T) <= LS_MAX_SLOT_BYTES;
+    if (T > LS_MAX_TOKENS || T * c.top_k > LS_MAX_ASSIGN || slot_bytes(c, T) > LS_MAX_SLOT_BYTES)
+        return false;
+    // The shared expert multiplies every weight with all T rows on the CUDA cores; with a large
+    // shared expert and more than one row that falls behind the weight stream, and the kernel
+    // chain (tensor cores) is the faster path (measured crossover).
+    return T == 1 || (size_t)T * c.shared_inter * c.hidden <= LS_SHARED_WORK_MAX;
 }
 
 // the largest T' <= T the one-launch kernel takes (0: none)
@@ -920,10 +964,10 @@ cudaError_t launch_layer_small(const moe_config_t &c, const moe_weights_t &w, co
     a.epoch = epoch;
     a.wait_us = (int)(LS_WAIT_NS / 1000ull);
     a.logit_chunks = (c.hidden + LS_LOGIT_CHUNK - 1) / LS_LOGIT_CHUNK;
-    a.chunks_r = down_chunks(c.inter);
-    a.chunk_r = down_chunk_cols(c.inter);
-    a.chunks_s = down_chunks(c.shared_inter);
-    a.chunk_s = down_chunk_cols(c.shared_inter);
+    a.chunks_r = down_chunks(c, c.inter);
+    a.chunk_r = down_chunk_cols(c, c.inter);
+    a.chunks_s = down_chunks(c, c.shared_inter);
+    a.chunk_s = down_chunk_cols(c, c.shared_inter);
     const size_t smem = slot_bytes(c, T);
     const int E = c.n_experts;
     if (E <= 32)
