@@ -137,6 +137,27 @@ def test_few_tokens_take_one_launch():
     assert api.moe_last_launch_count() > 1
 
 
+def test_one_workspace_serves_calls_of_every_size_in_turn():
+    """The one-launch kernel's barrier word and counters live in the workspace and are never
+    cleared: each call tags them with its own epoch.  Calls of one to five tokens (the last on
+    the kernel chain) alternate on ONE workspace, which starts out filled with a byte pattern;
+    every call must reproduce what a fresh workspace gives, and the status stays clear."""
+    from paper_2505_19645_b200 import api
+
+    shape = wl.small_shape("reuse", 512, 60, 4, 352, 1408, 0, 0, 1)
+    w = wl.make_weights(shape, 31, "cuda")
+    cfg, cw = api.make_config(shape), api.make_weights(w)
+    xs = {T: wl.make_tokens(shape, T, 40 + T, "cuda") for T in (1, 2, 3, 4, 5)}
+    want = {T: run_gpu_layer(shape, w, xs[T], T, 0)[0] for T in xs}
+    ws = torch.full((api.moe_workspace_bytes(cfg, 5),), 0xA5, dtype=torch.uint8, device="cuda")
+    for rep in range(6):
+        for T in (1, 4, 5, 2, 3, 1):
+            out = torch.empty_like(xs[T])
+            api.moe_verify_layer(cfg, cw, xs[T], T, 0, out, ws)
+            assert torch.equal(out, want[T]), (rep, T)
+    api.moe_check(ws)
+
+
 def test_kernel_chain_on_the_same_few_tokens():
     """The same cases with the one-launch kernel switched off (a test hook read once per
     process, hence the child process)."""
