@@ -570,8 +570,10 @@ def main():
     # ---- dominant kernel (gate/up) with its own event pair ----------------------------
     _, kern_ms = runner.time_steps(x, B, gamma, args.steps, 3, stage="gate_up")
     k_ms = sum(kern_ms) / len(kern_ms)
-    gu_bytes = gate_up_bytes(shape, T, n_act)
-    gu_flops = gate_up_flops(shape, T)
+    # one to four tokens may run as a single launch: the stage events then bracket the whole layer
+    whole_layer = launches_per_step == 1
+    gu_bytes = layer_bytes(shape, T, n_act) if whole_layer else gate_up_bytes(shape, T, n_act)
+    gu_flops = layer_flops(shape, T) if whole_layer else gate_up_flops(shape, T)
     t_mem = gu_bytes / (peaks["hbm_gbs"] * 1e9)
     t_flop = gu_flops / (peaks["bf16_tflops"] * 1e12)
     if t_mem >= t_flop:
@@ -583,7 +585,8 @@ def main():
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],
                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"]}
     roofline.update({"traffic": recorded_traffic(workload_name(args)),
-                     "kernel": "ffn_fused_kernel<gate/up + SwiGLU>",
+                     "kernel": ("layer_small_kernel (whole layer in one launch)" if whole_layer
+                                else "ffn_fused_kernel<gate/up + SwiGLU>"),
                      "kernel_ms": k_ms, "algorithmic_bytes": gu_bytes,
                      "peak_source": peaks["source"]})
 
