@@ -390,13 +390,19 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
         const bool probe_ = g_probe.stage == MOE_STAGE_GATE_UP;
         if (probe_ && cudaEventRecord(g_probe.start, s) != cudaSuccess)
             return MOE_ERR_CUDA;
-        if (launch_layer_small(*cfg, *w, xb, T, static_cast<__nv_bfloat16 *>(out), base, L, s) !=
-            cudaSuccess)
+        const cudaError_t err =
+            launch_layer_small(*cfg, *w, xb, T, static_cast<__nv_bfloat16 *>(out), base, L, s);
+        if (err == cudaSuccess) {
+            if (probe_ && cudaEventRecord(g_probe.stop, s) != cudaSuccess)
+                return MOE_ERR_CUDA;
+            g_last_launches = 1;
+            return copy_debug_out(*cfg, T, dbg, base, L, s);
+        }
+        // a context that cannot hold one CTA per SM at once (SMs set aside for others) refuses
+        // the cooperative launch: nothing was enqueued, the kernel sequence below serves the call
+        if (err != cudaErrorCooperativeLaunchTooLarge)
             return MOE_ERR_CUDA;
-        if (probe_ && cudaEventRecord(g_probe.stop, s) != cudaSuccess)
-            return MOE_ERR_CUDA;
-        g_last_launches = 1;
-        return copy_debug_out(*cfg, T, dbg, base, L, s);
+        (void)cudaGetLastError();
     }
     float *logits = reinterpret_cast<float *>(base + L.logits);
     int32_t *topk_idx = reinterpret_cast<int32_t *>(base + L.topk_idx);
