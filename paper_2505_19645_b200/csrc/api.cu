@@ -426,15 +426,16 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
     } arm;
     const PlanView plan = plan_view(base, L, ffn_segment_rows(*cfg, T));
     int32_t *status = reinterpret_cast<int32_t *>(base + L.status);
+    int logit_chunks = 0;  // > 0: the logits are still partial sums per k chunk (summed by the top-k)
     if (router_logits_tc_applies(*cfg, T)) {
         const bool probe_ = g_probe_armed && g_probe.stage == MOE_STAGE_ROUTER_LOGITS;
         if (probe_ && cudaEventRecord(g_probe.start, s) != cudaSuccess)
             return MOE_ERR_CUDA;
-        if (launch_router_logits_tc(*cfg, *w, xb, T, logits, gated ? shared_scale : nullptr,
+        if (launch_router_logits_tc(*cfg, *w, xb, T,
                                     reinterpret_cast<__nv_bfloat16 *>(base + L.rl_planes),
                                     reinterpret_cast<float *>(base + L.rl_partial), s,
                                     plan.done_shared, max_shared_segments(T), status,
-                                    &launches) != cudaSuccess)
+                                    &launches, &logit_chunks) != cudaSuccess)
             return MOE_ERR_CUDA;
         if (probe_ && cudaEventRecord(g_probe.stop, s) != cudaSuccess)
             return MOE_ERR_CUDA;
@@ -452,7 +453,14 @@ moe_status_t moe_verify_layer(const moe_config_t *cfg, const moe_weights_t *w, c
                                            perm, inv_perm, active, n_active, status, plan,
                                            reinterpret_cast<__nv_bfloat16 *>(base + L.x_sorted), s));
     } else {
-        MOE_STAGE(MOE_STAGE_ROUTE_TOPK, launch_route_topk(*cfg, logits, T, topk_idx, topk_w, s));
+        if (logit_chunks > 0)
+            MOE_STAGE(MOE_STAGE_ROUTE_TOPK,
+                      launch_route_topk_sum(*cfg, reinterpret_cast<const float *>(base + L.rl_partial),
+                                            logit_chunks, cfg->n_experts + (gated ? 1 : 0),
+                                            w->router_bias, T, logits, gated ? shared_scale : nullptr,
+                                            topk_idx, topk_w, s));
+        else
+            MOE_STAGE(MOE_STAGE_ROUTE_TOPK, launch_route_topk(*cfg, logits, T, topk_idx, topk_w, s));
         MOE_STAGE(MOE_STAGE_PERMUTE,
                   launch_permute(*cfg, topk_idx, T, counts, offsets, perm, inv_perm, active,
                                  n_active, s, &plan, status));

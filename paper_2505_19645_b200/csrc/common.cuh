@@ -187,15 +187,22 @@ cudaError_t launch_router_logits(const moe_config_t &c, const moe_weights_t &w,
                                  const __nv_bfloat16 *x, int T, float *logits,
                                  float *shared_scale, cudaStream_t s, int32_t *zero = nullptr,
                                  int zero_n = 0, int32_t *status = nullptr);
-// The same on tcgen05 for large batches (router_logits_tc.cu): three launches (split of the fp32
-// rows into bf16 planes, the contraction, the sum of its k chunks); planes / partial are the
-// workspace regions of router_tc_plane_bytes / router_tc_partial_bytes.
+// The same on tcgen05 for large batches (router_logits_tc.cu): two launches (split of the fp32
+// rows into bf16 planes, the contraction); planes / partial are the workspace regions of
+// router_tc_plane_bytes / router_tc_partial_bytes.  The logits are left as partial sums
+// [*chunks][T][E (+1 with the shared gate's row)] in `partial`: launch_route_topk_sum adds them.
 cudaError_t launch_router_logits_tc(const moe_config_t &c, const moe_weights_t &w,
-                                    const __nv_bfloat16 *x, int T, float *logits, float *shared_scale,
-                                    __nv_bfloat16 *planes, float *partial, cudaStream_t s,
-                                    int32_t *zero, int zero_n, int32_t *status, int *launches);
+                                    const __nv_bfloat16 *x, int T, __nv_bfloat16 *planes,
+                                    float *partial, cudaStream_t s, int32_t *zero, int zero_n,
+                                    int32_t *status, int *launches, int *chunks);
 cudaError_t launch_route_topk(const moe_config_t &c, const float *logits, int T, int32_t *idx,
                               float *wts, cudaStream_t s);
+// the same from partial logits [chunks][T][R] (R = E, or E + 1 with the shared gate's row last):
+// sums the chunks in chunk order, adds the bias, writes logits [T,E] (and shared_scale [T] if not
+// null) and selects
+cudaError_t launch_route_topk_sum(const moe_config_t &c, const float *partial, int chunks, int R,
+                                  const float *bias, int T, float *logits, float *shared_scale,
+                                  int32_t *idx, float *wts, cudaStream_t s);
 cudaError_t launch_permute(const moe_config_t &c, const int32_t *idx, int T, int32_t *counts,
                            int32_t *offsets, int32_t *perm, int32_t *inv_perm, int32_t *active,
                            int32_t *n_active, cudaStream_t s, const PlanView *plan = nullptr,

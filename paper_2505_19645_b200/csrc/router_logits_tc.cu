@@ -5,12 +5,13 @@
 // with fp32-level accuracy from bf16 instructions: every fp32 router row is split once per call
 // into three bf16 rows  w = hi + mid + lo  (each remainder is exact in fp32, so the three carry
 // 24 mantissa bits; the bf16 token values are exact) and the three products are accumulated in
-// the same fp32 accumulator in TMEM.  Three kernels:
+// the same fp32 accumulator in TMEM.  Two kernels here, and the first step of a third:
 //   split   w_router (and the bf16 gate vector) -> planes [3][R][H] bf16, R = E (+1)
 //   gemm    one CTA per (256 tokens, 256 router rows, k chunk): TMA -> shared-memory rings ->
 //           tcgen05.mma (router rows as M, two blocks of 128; tokens as N) -> partial sums
 //           [S][T][R] fp32
-//   reduce  sums the S partial planes in a fixed order, adds the bias, applies the sigmoid
+//   sum     route_topk_sum_kernel (router.cu): the warp that ranks a token's logits first adds its
+//           S partial rows in chunk order, adds the bias and applies the gate's sigmoid
 // The reduction over H is cut into S chunks so that about one CTA per SM has work even when
 // there are only a dozen token tiles; the partial planes are summed in chunk order, so the
 // logits do not depend on timing.  Used for large batches (router_logits_tc_applies), where the
@@ -33,7 +34,7 @@ constexpr int RT_B_BYTES = RT_TOKENS * 128;
 constexpr int RT_MAX_SPLIT = 16;
 constexpr int RT_SMEM = RT_A_SLOTS * RT_A_BYTES + RT_B_SLOTS * RT_B_BYTES + 1024;
 
-// From about 128 K logits on the mma.sync kernel takes longer than the three launches here
+// From about 128 K logits on the mma.sync kernel takes longer than the launches here
 // (measured: 256 experts from 512 tokens, 64 experts from 2048 tokens).
 bool router_logits_tc_applies(const moe_config_t &c, int T)
 {
@@ -123,29 +124,6 @@ router_split_kernel(const float *__restrict__ w_router, const __nv_bfloat16 *__r
         *reinterpret_cast<uint4 *>(planes + at) = hi;
         *reinterpret_cast<uint4 *>(planes + plane + at) = mid;
         *reinterpret_cast<uint4 *>(planes + 2 * plane + at) = lo;
-    }
-}
-
-// ---- reduce: partial planes -> logits ---------------------------------------------------------
-
-__global__ void __launch_bounds__(256)
-router_reduce_kernel(const float *__restrict__ partial, int S, int T, int E, int R,
-                     const float *__restrict__ bias, float *__restrict__ logits,
-                     float *__restrict__ shared_scale)
-{
-    griddep_launch();
-    griddep_wait();  // the partial sums come from the preceding kernel
-    const size_t n = (size_t)T * R, plane = n;
-    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n;
-         i += (size_t)gridDim.x * blockDim.x) {
-        const int t = (int)(i / R), e = (int)(i - (size_t)t * R);
-        float v = 0.f;
-        for (int s = 0; s < S; ++s)  // chunk order: the sum does not depend on scheduling
-            v += partial[(size_t)s * plane + i];
-        if (e < E)
-            logits[(size_t)t * E + e] = bias ? v + bias[e] : v;
-        else if (shared_scale != nullptr)
-            shared_scale[t] = 1.0f / (1.0f + expf(-v));
     }
 }
 
@@ -354,14 +332,11 @@ router_logits_tc_kernel(const RouterTcArgs args, const __grid_constant__ RouterT
 // ---- host -----------------------------------------------------------------------------------------
 
 cudaError_t launch_router_logits_tc(const moe_config_t &c, const moe_weights_t &w,
-                                    const __nv_bfloat16 *x, int T, float *logits, float *shared_scale,
-                                    __nv_bfloat16 *planes, float *partial, cudaStream_t s,
-                                    int32_t *zero, int zero_n, int32_t *status, int *launches)
+                                    const __nv_bfloat16 *x, int T, __nv_bfloat16 *planes,
+                                    float *partial, cudaStream_t s, int32_t *zero, int zero_n,
+                                    int32_t *status, int *launches, int *chunks)
 {
-    const bool gate_row = shared_scale != nullptr && c.shared_gate && c.shared_inter > 0;
     const int E = c.n_experts, R = router_rows(c), H = c.hidden;
-    // the planes always hold router_rows() rows; without an output for the gate its row is
-    // computed and dropped
     cudaError_t err = launch_pdl(router_split_kernel, dim3(2 * sm_count()), dim3(256), 0, s, w.w_router,
                                  static_cast<const __nv_bfloat16 *>(w.w_shared_gate), E, R, H, planes,
                                  zero, zero_n, status);
@@ -434,16 +409,7 @@ cudaError_t launch_router_logits_tc(const moe_config_t &c, const moe_weights_t &
         return err;
     ++*launches;
 
-    const size_t n = (size_t)T * R;
-    size_t blocks = (n + 255) / 256;
-    if (blocks > (size_t)sm_count() * 8)
-        blocks = (size_t)sm_count() * 8;
-    err = launch_pdl(router_reduce_kernel, dim3((unsigned)blocks), dim3(256), 0, s,
-                     static_cast<const float *>(partial), a.split, T, E, R, w.router_bias, logits,
-                     gate_row ? shared_scale : nullptr);
-    if (err != cudaSuccess)
-        return err;
-    ++*launches;
+    *chunks = a.split;  // the caller's top-k kernel sums them
     return cudaSuccess;
 }
 
