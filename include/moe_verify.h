@@ -229,11 +229,13 @@ moe_status_t moe_check(void *ws, void *stream);
 
 /* Self-test of the failure path (no counterpart in the paper).  Every wait inside the kernels is
  * bounded; when one gives up, the kernel raises the workspace's status word and returns, and
- * moe_check reports MOE_ERR_TIMEOUT while the context stays usable.  This call enqueues one tiny
- * kernel that runs exactly that wait -- the one the down projection uses for the progress
- * counters of the gate/up pass -- on a word nothing ever sets, with a limit of limit_us
- * microseconds (1 .. 1000000).  ws: any workspace of at least 256 bytes; its status word is
- * overwritten.  Returns at once; the outcome is read with moe_check(ws, stream). */
+ * moe_check reports MOE_ERR_TIMEOUT while the context stays usable.  This call enqueues two tiny
+ * kernels that run exactly those waits -- the one the down projection uses for the progress
+ * counters of the gate/up pass, then the one the one-launch layer of a few tokens uses for its
+ * grid barrier and per-expert counters -- each on a word nothing ever advances, each with a limit
+ * of limit_us microseconds (1 .. 1000000).  ws: any workspace of at least 256 bytes; its status
+ * word is overwritten (the fourth 32-bit word of ws reads 1 once the second wait has given up).
+ * Returns at once; the outcome is read with moe_check(ws, stream). */
 moe_status_t moe_selftest_wait_limit(void *ws, int32_t limit_us, void *stream);
 
 /* Measurement aid (no counterpart in the paper; its Sec. 3.3 model attributes the layer's

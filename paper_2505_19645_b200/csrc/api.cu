@@ -512,6 +512,7 @@ moe_status_t moe_selftest_wait_limit(void *ws, int32_t limit_us, void *stream)
     int launches = 0;
     MOE_TRY_LAUNCH(launch_wait_limit_selftest(status, status + 2, limit_us,
                                               static_cast<cudaStream_t>(stream)));
+    MOE_TRY_LAUNCH(launch_tagged_wait_selftest(status, limit_us, static_cast<cudaStream_t>(stream)));
     return MOE_OK;
 }
 

@@ -233,6 +233,9 @@ cudaError_t launch_route_group_small(const moe_config_t &c, const float *logits,
 // one bounded wait on a word nothing sets (moe_selftest_wait_limit)
 cudaError_t launch_wait_limit_selftest(int32_t *status, int32_t *never_set, int limit_us,
                                        cudaStream_t s);
+// the same for the wait of the one-launch layer's counters; word [3] of the status region is set
+// to 1 when that wait gave up
+cudaError_t launch_tagged_wait_selftest(int32_t *status, int limit_us, cudaStream_t s);
 // token rows in sorted order (the token operand of the routed gate/up tiles)
 cudaError_t launch_gather_rows(const moe_config_t &c, const __nv_bfloat16 *x, const int32_t *perm,
                                int T, __nv_bfloat16 *x_sorted, cudaStream_t s);

@@ -49,6 +49,7 @@ constexpr int LS_DOWN_ROWS = 4;       // output features per down-projection wor
 constexpr int LS_SLOT_FLOATS = LS_DOWN_ROWS * LS_MAX_TOKENS;  // partial sums of one such item
 constexpr size_t LS_MAX_SLOT_BYTES = 160u << 10;
 constexpr uint64_t LS_WAIT_NS = 1000ull * 1000ull * 1000ull;
+constexpr int LS_SELFTEST_WORD = 4;  // int32 index there of the word the wait self-test waits on
 constexpr int LS_BARRIER_WORD = 8;  // int32 index of the grid barrier's word inside the status region
 constexpr size_t LS_UNIT_WORD_BYTES = 512;  // the units' counters lead the partial-logit region
 
@@ -781,6 +782,30 @@ __global__ void __launch_bounds__(LS_THREADS, 1) layer_small_kernel(const SmallA
         packed.y = *reinterpret_cast<const uint32_t *>(&hi);
         *reinterpret_cast<uint2 *>(a.out + (size_t)t * H + f0) = packed;
     }
+}
+
+// ---- self-test of the bounded wait -------------------------------------------------------------
+
+// Waits, with the given limit, for a counter that nothing advances: the wait of the one-launch
+// layer (grid barrier, unit counters) must give up, raise the status word and return.  Word [3] of
+// the status region records that it did.
+__global__ void tagged_wait_selftest_kernel(int32_t *status, unsigned long long *never_reached,
+                                            int limit_us)
+{
+    if (threadIdx.x == 0) {
+        *never_reached = 0ull;
+        status[3] = 0;
+        __threadfence();
+        const bool reached = tagged_wait(never_reached, 0xffffffffu, 1u, status, limit_us);
+        status[3] = reached ? 0 : 1;
+    }
+}
+
+cudaError_t launch_tagged_wait_selftest(int32_t *status, int limit_us, cudaStream_t s)
+{
+    tagged_wait_selftest_kernel<<<1, 32, 0, s>>>(
+        status, reinterpret_cast<unsigned long long *>(status + LS_SELFTEST_WORD), limit_us);
+    return cudaGetLastError();
 }
 
 // ---- host -------------------------------------------------------------------------------------

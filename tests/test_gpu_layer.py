@@ -230,7 +230,8 @@ def test_layer_parity_with_plain_stream_ordering():
 
 def test_wait_limit_expiry_is_reported_and_the_context_stays_usable():
     """Every wait inside the kernels has a limit.  The self-test runs the down pass's wait for
-    a progress counter on a word nothing sets: it gives up after its limit, the kernel raises
+    a progress counter, and the one-launch layer's wait for its grid-wide counters, each on a
+    word nothing advances: each gives up after its limit, the kernel raises
     the workspace's status word and returns, moe_check reports MOE_ERR_TIMEOUT, nothing
     faults, and the same workspace serves a correct layer call right after.  The word is
     sticky: a layer call enqueued behind the failed wait does not erase the report, and the
@@ -251,8 +252,13 @@ def test_wait_limit_expiry_is_reported_and_the_context_stays_usable():
         api.moe_check(ws)
     waited = time.perf_counter() - t0
     assert err.value.status == 5  # MOE_ERR_TIMEOUT
-    assert 0.015 < waited < 1.0
+    assert 0.035 < waited < 1.0   # two waits of 20 ms: the tile kernels' and the one-launch layer's
+    assert int(ws[12:16].view(torch.int32).item()) == 1   # the second wait gave up too
     api.moe_check(ws)   # reported once
+    x3 = wl.make_tokens(shape, 3, 268, "cuda")
+    out3, _ = run_gpu_layer(shape, w, x3, 3, 0, ws=ws)   # the one-launch layer on the same workspace
+    ref3, _ = run_gpu_layer(shape, w, x3, 3, 0)
+    assert torch.equal(out3, ref3)
     # a failure in an earlier call of a queue is still seen after later calls
     out = torch.empty_like(x)
     api.moe_selftest_wait_limit(ws, 2000)
