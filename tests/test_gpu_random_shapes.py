@@ -54,3 +54,27 @@ def test_random_shapes_match_the_oracle(seed):
             check_layer_against_oracle(shape, w, x, T, 0)
         except AssertionError as e:
             raise AssertionError("case %d (%s): %s" % (n, name, e)) from e
+
+
+def test_random_shapes_of_a_few_tokens():
+    """One to four tokens: the one-launch kernel (where T * top_k <= 32, else the kernel chain),
+    with intermediate sizes that cut the down projection into one to three column chunks."""
+    rng = random.Random(14)
+    for n in range(160):
+        H, E, k, I, Is, score, renorm, sgate, zipf, _ = draw_case(rng)
+        T = rng.randint(1, 4)
+        if n % 3 == 0:
+            I = 32 * rng.choice([65, 100, 136, 150])      # 2080 .. 4800 columns
+        if n % 5 == 0 and Is:
+            Is = 32 * rng.choice([70, 129, 200])          # 2240 .. 6400 columns
+        if E * I * H * 6 > 1_000_000_000:
+            continue
+        name = "few-H%d-E%d-k%d-I%d-Is%d-s%d-r%d-g%d-z%s-T%d" % (H, E, k, I, Is, score, renorm,
+                                                              sgate, zipf, T)
+        shape = wl.small_shape(name, H, E, k, I, Is, score, renorm, sgate)
+        w = wl.make_weights(shape, 14000 + n, "cuda", zipf_s=zipf)
+        x = wl.make_tokens(shape, T, 15000 + n, "cuda")
+        try:
+            check_layer_against_oracle(shape, w, x, T, 0)
+        except AssertionError as e:
+            raise AssertionError("case %d (%s): %s" % (n, name, e)) from e
